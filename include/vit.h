@@ -1,0 +1,176 @@
+/*
+ * vit.h — C boundary of the ViT pipeline-stage forward library for NVIDIA B200 (sm_100a).
+ *
+ * The library computes the forward pass of one pipeline stage: a contiguous range of layers
+ * [layer_begin, layer_end) of a pre-LN Vision Transformer encoder applied to one microbatch of
+ * activations, plus the two book-ends (patch embedding before the first stage, classification
+ * head after the last) and a stage runner that issues microbatches on CUDA streams.
+ *
+ * Conventions for every entry point
+ *   - All functions return an int status: VIT_OK (0) or a negative VIT_ERR_* code.  Arguments
+ *     are validated on the host before anything is launched; a failed call launches nothing.
+ *   - "dev" pointers are device memory owned by the caller (for example the data_ptr() of a
+ *     PyTorch tensor) and must stay alive until the stream has drained.  They must be 16-byte
+ *     aligned.  "host" pointers are ordinary (preferably pinned) host memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls are
+ *     asynchronous on that stream, allocate nothing and never synchronise the host, except
+ *     where stated.
+ *   - Activations are row-major [microbatch, T, H] (T = patches + 1 class token, H = hidden).
+ *     Their element type is the model's activation type: bf16 when config.dtype == VIT_BF16
+ *     (bf16 operands, fp32 accumulation), fp32 when config.dtype == VIT_FP32.
+ *   - A workspace must not be shared by two calls that may overlap on the GPU.
+ *   - A handle may be used from several host threads at once with distinct streams and
+ *     workspaces; parameters are read-only after vit_create.
+ */
+#ifndef VIT_B200_H
+#define VIT_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  VIT_OK = 0,
+  VIT_ERR_INVALID_ARG = -1, /* null or misaligned pointer, microbatch < 1 or > max_microbatch */
+  VIT_ERR_RANGE = -2,       /* not 0 <= layer_begin < layer_end <= layers (empty range is an error) */
+  VIT_ERR_CONFIG = -3,      /* inconsistent or unsupported model shape */
+  VIT_ERR_WORKSPACE = -4,   /* workspace smaller than the size query says */
+  VIT_ERR_CUDA = -5,        /* a CUDA runtime/driver call or a launch failed */
+  VIT_ERR_TIMEOUT = -6,     /* a bounded wait inside a kernel gave up (device status word) */
+  VIT_ERR_NO_DEVICE = -7    /* no sm_100 device / driver available */
+};
+
+enum { VIT_BF16 = 0, VIT_FP32 = 1 };
+
+typedef struct vit_config {
+  int32_t image_size;     /* pixels per side, e.g. 224 */
+  int32_t patch_size;     /* 16 or 14; must divide image_size */
+  int32_t channels;       /* 3 */
+  int32_t hidden;         /* H, multiple of 64 */
+  int32_t layers;         /* L */
+  int32_t heads;          /* H / heads must be a multiple of 16 and <= 128 */
+  int32_t mlp_dim;        /* F, multiple of 64 */
+  int32_t num_classes;
+  float   ln_eps;         /* LayerNorm epsilon (inside the square root) */
+  int32_t dtype;          /* VIT_BF16 or VIT_FP32 */
+  int32_t max_microbatch; /* largest microbatch any call will use */
+} vit_config;
+
+typedef struct vit_handle vit_handle; /* opaque */
+
+/* Number of fp32 values in the host parameter blob for this configuration (0 if the
+ * configuration is invalid).  Blob layout, tensors back to back, matrices [out, in] row-major:
+ *   patch.W [H, C*P*P] (column = c*P*P + i*P + j), patch.b [H], cls [H], pos [T, H],
+ *   per layer: ln1.g ln1.b Wqkv[3H,H] bqkv[3H] Wo[H,H] bo[H] ln2.g ln2.b W1[F,H] b1[F] W2[H,F] b2[H],
+ *   lnf.g [H], lnf.b [H], head.W [classes, H], head.b [classes].
+ * Wqkv rows [0,H) produce Q, [H,2H) K, [2H,3H) V; head h owns rows h*d..(h+1)*d of each. */
+size_t vit_param_count(const vit_config* cfg);
+
+/* Bytes of scratch one call of vit_patch_embed / vit_run_stage / vit_head needs for
+ * `microbatch` images (the maximum over the three).  0 if arguments are invalid. */
+size_t vit_workspace_bytes(const vit_config* cfg, int microbatch);
+
+/* Bytes of scratch one stream of vit_run_pipeline[_host] needs for `microbatch` images:
+ * the stage scratch above plus the token buffer and pixel/logit staging. */
+size_t vit_pipeline_workspace_bytes(const vit_config* cfg, int microbatch);
+
+/* Creates a model instance on the current CUDA device.
+ * The transformer to partition is given to the system as a configuration plus its weights
+ * (paper Section 3.1: the model configuration is the partitioner's input; Section 4: the
+ * models are standard ViT definitions).
+ *   host_params: host, fp32 blob in the layout above, n_params == vit_param_count(cfg).
+ *     In bf16 mode matrices are rounded to bf16 (nearest even) on upload; vectors stay fp32.
+ * Allocates device memory for the parameters (freed by vit_destroy), synchronises.
+ * Errors: INVALID_ARG, CONFIG, NO_DEVICE, CUDA. */
+int vit_create(const vit_config* cfg, const float* host_params, size_t n_params, vit_handle** out);
+
+/* Frees the handle and the device memory it allocated.  Synchronises the device. */
+int vit_destroy(vit_handle* h);
+
+/* Embedding book-end (paper Section 4: inputs pass an embedding layer that gives them the
+ * uniform dimension the transformer layers expect).
+ *   pixels: dev, fp32 [microbatch, C, S, S] (NCHW).
+ *   tokens_out: dev, activations [microbatch, T, H].  Token 1 + py*(S/P) + px is
+ *     patch.W . vec(patch(py,px)) + patch.b + pos[token]; token 0 is cls + pos[0].
+ *   ws: dev scratch of at least vit_workspace_bytes(cfg, microbatch). */
+int vit_patch_embed(vit_handle* h, int microbatch, const float* pixels, void* tokens_out,
+                    void* ws, size_t ws_bytes, void* stream);
+
+/* One pipeline stage T_i (paper Section 3.1: the model is split into parts T_1..T_k of
+ * consecutive layers, the output of stage i is the input of stage i+1, and
+ * Y = T_k(...T_1(X))).  Applies layers [layer_begin, layer_end) to `in`, writes `out`.
+ * Each layer is x += Wo.attention(LN1(x).Wqkv^T + bqkv) + bo;  x += W2.gelu(W1.LN2(x) + b1) + b2
+ * (Section 2.1: self-attention, MLP, two layer normalisations, residual connections).
+ *   in, out: dev, activations [microbatch, T, H]; in == out is allowed (in place), any other
+ *     overlap is INVALID_ARG.
+ * Running [a,b) then [b,c) gives bit-identical results to one call on [a,c). */
+int vit_run_stage(vit_handle* h, int layer_begin, int layer_end, int microbatch,
+                  const void* in, void* out, void* ws, size_t ws_bytes, void* stream);
+
+/* Classification book-end (paper Section 3.1: the device of the final stage produces the
+ * final result; Section 4: the task is image classification).  Final LayerNorm of each image's
+ * class token, then logits = f . head.W^T + head.b.
+ *   tokens: dev, activations [microbatch, T, H];  logits: dev, fp32 [microbatch, classes]. */
+int vit_head(vit_handle* h, int microbatch, const void* tokens, float* logits,
+             void* ws, size_t ws_bytes, void* stream);
+
+/* Stage runner (paper Section 2.1/3.1: the minibatch is split into equal microbatches that
+ * flow through the stages in order).  Splits `batch` images into microbatches of `microbatch`
+ * (the last may be smaller), and for microbatch m issues, on streams[m % n_streams]:
+ * patch embed, every stage in order (stage s covers stage_layers[s] layers; the counts must
+ * sum to L), head.  A microbatch never changes stream, so stream order carries the
+ * stage-to-stage dependency; different microbatches overlap across streams.
+ *   pixels: dev fp32 [batch, C, S, S];  logits: dev fp32 [batch, classes].
+ *   ws_per_stream[i]: dev scratch of at least vit_pipeline_workspace_bytes(cfg, microbatch).
+ * Does not synchronise; the caller waits on the streams. */
+int vit_run_pipeline(vit_handle* h, const int32_t* stage_layers, int n_stages, int batch,
+                     int microbatch, const float* pixels, float* logits,
+                     void* const* ws_per_stream, size_t ws_bytes, void* const* streams,
+                     int n_streams);
+
+/* Same as vit_run_pipeline with HOST pixels and logits: each microbatch's pixels are copied to
+ * the device, and its logits back, on that microbatch's stream (copies are asynchronous only
+ * if the host memory is pinned).  Does not synchronise. */
+int vit_run_pipeline_host(vit_handle* h, const int32_t* stage_layers, int n_stages, int batch,
+                          int microbatch, const float* host_pixels, float* host_logits,
+                          void* const* ws_per_stream, size_t ws_bytes, void* const* streams,
+                          int n_streams);
+
+/* Synchronises `stream`, then returns and clears the device status word: VIT_OK, or
+ * VIT_ERR_TIMEOUT if a bounded wait in a kernel gave up since the last check, or VIT_ERR_CUDA
+ * if the stream reported an error. */
+int vit_check_status(vit_handle* h, void* stream);
+
+/* Number of kernels this handle has launched so far (host counter). */
+uint64_t vit_launch_count(const vit_handle* h);
+
+const char* vit_status_string(int status);
+
+/* ---- single operations, exposed so that each kernel can be checked on its own ------------
+ * All pointers dev; `dtype` selects the bf16 or fp32 kernel family as in vit_config.
+ * They need a handle only for the device status word and the launch counter. */
+
+/* y[r,:] = (x[r,:] - mean) / sqrt(var + eps) * gain + shift, biased variance, rows x cols.
+ * x, y: activations; gain, shift: fp32 [cols]. */
+int vit_op_layernorm(vit_handle* h, int dtype, int rows, int cols, const void* x,
+                     const float* gain, const float* shift, float eps, void* y, void* stream);
+
+/* out = epilogue(a[M,K] . w[N,K]^T + bias[N]); a, w, out, residual in the activation type,
+ * bias fp32.  epilogue: 0 = none, 1 = erf-GELU, 2 = add residual[M,N] (residual may equal out).
+ * bf16 family: K % 8 == 0 and N % 8 == 0. */
+int vit_op_linear(vit_handle* h, int dtype, int M, int N, int K, const void* a, const void* w,
+                  const float* bias, int epilogue, const void* residual, void* out, void* stream);
+
+/* Multi-head self-attention for `images` sequences of T tokens: qkv [images*T, 3*heads*d]
+ * (column blocks Q, K, V; head-major inside each), out [images*T, heads*d];
+ * out_h = softmax_rows(Q_h K_h^T / sqrt(d)) V_h. */
+int vit_op_attention(vit_handle* h, int dtype, int images, int T, int heads, int d,
+                     const void* qkv, void* out, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VIT_B200_H */

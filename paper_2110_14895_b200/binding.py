@@ -1,0 +1,279 @@
+"""ctypes binding of libvit_b200.so: the same entry points as include/vit.h, argument
+marshalling only.  Every step of the forward pass runs in the library's CUDA kernels; there is
+no fallback: if the library is missing or a call fails, an exception is raised.
+
+PyTorch appears here only as the owner of device memory and streams (`data_ptr()`,
+`torch.cuda.Stream.cuda_stream`).
+"""
+import ctypes
+import os
+from ctypes import (POINTER, Structure, byref, c_char_p, c_float, c_int, c_int32, c_size_t,
+                    c_uint64, c_void_p)
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libvit_b200.so")
+
+VIT_OK = 0
+VIT_ERR_INVALID_ARG, VIT_ERR_RANGE, VIT_ERR_CONFIG, VIT_ERR_WORKSPACE = -1, -2, -3, -4
+VIT_ERR_CUDA, VIT_ERR_TIMEOUT, VIT_ERR_NO_DEVICE = -5, -6, -7
+VIT_BF16, VIT_FP32 = 0, 1
+
+EXPORTS = [
+    "vit_param_count", "vit_workspace_bytes", "vit_pipeline_workspace_bytes", "vit_create",
+    "vit_destroy", "vit_patch_embed", "vit_run_stage", "vit_head", "vit_run_pipeline",
+    "vit_run_pipeline_host", "vit_check_status", "vit_launch_count", "vit_status_string",
+    "vit_op_layernorm", "vit_op_linear", "vit_op_attention",
+]
+
+
+class VitConfig(Structure):
+    _fields_ = [
+        ("image_size", c_int32), ("patch_size", c_int32), ("channels", c_int32),
+        ("hidden", c_int32), ("layers", c_int32), ("heads", c_int32), ("mlp_dim", c_int32),
+        ("num_classes", c_int32), ("ln_eps", c_float), ("dtype", c_int32),
+        ("max_microbatch", c_int32),
+    ]
+
+
+class VitError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+_lib = None
+
+
+def lib():
+    """Loads the shared library (once).  Fails loudly when it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2110_14895_b200.build`")
+    L = ctypes.CDLL(LIB_PATH)
+    P = POINTER
+    L.vit_param_count.restype = c_size_t
+    L.vit_param_count.argtypes = [P(VitConfig)]
+    L.vit_workspace_bytes.restype = c_size_t
+    L.vit_workspace_bytes.argtypes = [P(VitConfig), c_int]
+    L.vit_pipeline_workspace_bytes.restype = c_size_t
+    L.vit_pipeline_workspace_bytes.argtypes = [P(VitConfig), c_int]
+    L.vit_create.restype = c_int
+    L.vit_create.argtypes = [P(VitConfig), c_void_p, c_size_t, P(c_void_p)]
+    L.vit_destroy.restype = c_int
+    L.vit_destroy.argtypes = [c_void_p]
+    L.vit_patch_embed.restype = c_int
+    L.vit_patch_embed.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    L.vit_run_stage.restype = c_int
+    L.vit_run_stage.argtypes = [c_void_p, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    L.vit_head.restype = c_int
+    L.vit_head.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    for f in (L.vit_run_pipeline, L.vit_run_pipeline_host):
+        f.restype = c_int
+        f.argtypes = [c_void_p, P(c_int32), c_int, c_int, c_int, c_void_p, c_void_p, P(c_void_p),
+                      c_size_t, P(c_void_p), c_int]
+    L.vit_check_status.restype = c_int
+    L.vit_check_status.argtypes = [c_void_p, c_void_p]
+    L.vit_launch_count.restype = c_uint64
+    L.vit_launch_count.argtypes = [c_void_p]
+    L.vit_status_string.restype = c_char_p
+    L.vit_status_string.argtypes = [c_int]
+    L.vit_op_layernorm.restype = c_int
+    L.vit_op_layernorm.argtypes = [c_void_p, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_void_p]
+    L.vit_op_linear.restype = c_int
+    L.vit_op_linear.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p]
+    L.vit_op_attention.restype = c_int
+    L.vit_op_attention.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p]
+    _lib = L
+    return L
+
+
+def status_string(status: int) -> str:
+    return lib().vit_status_string(status).decode()
+
+
+def _check(status, where):
+    if status != VIT_OK:
+        raise VitError(status, where)
+
+
+def make_config(shape, dtype=VIT_BF16, max_microbatch=1) -> VitConfig:
+    """`shape` is any object with image_size, patch_size, channels, hidden, layers, heads,
+    mlp_dim, num_classes, ln_eps attributes."""
+    return VitConfig(shape.image_size, shape.patch_size, shape.channels, shape.hidden, shape.layers,
+                     shape.heads, shape.mlp_dim, shape.num_classes, float(shape.ln_eps), int(dtype),
+                     int(max_microbatch))
+
+
+# ---- thin wrappers with the names of the C entry points (raw pointers as ints) ----------------
+def vit_param_count(cfg: VitConfig) -> int:
+    return lib().vit_param_count(byref(cfg))
+
+
+def vit_workspace_bytes(cfg: VitConfig, microbatch: int) -> int:
+    return lib().vit_workspace_bytes(byref(cfg), microbatch)
+
+
+def vit_pipeline_workspace_bytes(cfg: VitConfig, microbatch: int) -> int:
+    return lib().vit_pipeline_workspace_bytes(byref(cfg), microbatch)
+
+
+def vit_create(cfg: VitConfig, host_params: np.ndarray) -> int:
+    if host_params.dtype != np.float32 or not host_params.flags["C_CONTIGUOUS"]:
+        raise TypeError("host_params must be a contiguous float32 array")
+    h = c_void_p()
+    _check(lib().vit_create(byref(cfg), host_params.ctypes.data, host_params.size, byref(h)), "vit_create")
+    return h.value
+
+
+def vit_destroy(h: int) -> None:
+    _check(lib().vit_destroy(h), "vit_destroy")
+
+
+def vit_patch_embed(h, microbatch, pixels, tokens_out, ws, ws_bytes, stream=0):
+    _check(lib().vit_patch_embed(h, microbatch, pixels, tokens_out, ws, ws_bytes, stream), "vit_patch_embed")
+
+
+def vit_run_stage(h, layer_begin, layer_end, microbatch, inp, out, ws, ws_bytes, stream=0):
+    _check(lib().vit_run_stage(h, layer_begin, layer_end, microbatch, inp, out, ws, ws_bytes, stream),
+           "vit_run_stage")
+
+
+def vit_head(h, microbatch, tokens, logits, ws, ws_bytes, stream=0):
+    _check(lib().vit_head(h, microbatch, tokens, logits, ws, ws_bytes, stream), "vit_head")
+
+
+def _pipeline(fn, name, h, stage_layers, batch, microbatch, pixels, logits, ws_ptrs, ws_bytes, streams):
+    n = len(stage_layers)
+    sl = (c_int32 * n)(*stage_layers)
+    k = len(streams)
+    if len(ws_ptrs) != k:
+        raise ValueError("one workspace per stream")
+    wsa = (c_void_p * k)(*ws_ptrs)
+    sta = (c_void_p * k)(*streams)
+    _check(fn(h, sl, n, batch, microbatch, pixels, logits, wsa, ws_bytes, sta, k), name)
+
+
+def vit_run_pipeline(h, stage_layers, batch, microbatch, pixels, logits, ws_ptrs, ws_bytes, streams):
+    _pipeline(lib().vit_run_pipeline, "vit_run_pipeline", h, stage_layers, batch, microbatch, pixels,
+              logits, ws_ptrs, ws_bytes, streams)
+
+
+def vit_run_pipeline_host(h, stage_layers, batch, microbatch, host_pixels, host_logits, ws_ptrs,
+                          ws_bytes, streams):
+    _pipeline(lib().vit_run_pipeline_host, "vit_run_pipeline_host", h, stage_layers, batch, microbatch,
+              host_pixels, host_logits, ws_ptrs, ws_bytes, streams)
+
+
+def vit_check_status(h, stream=0) -> None:
+    _check(lib().vit_check_status(h, stream), "vit_check_status")
+
+
+def vit_launch_count(h) -> int:
+    return lib().vit_launch_count(h)
+
+
+def vit_op_layernorm(h, dtype, rows, cols, x, gain, shift, eps, y, stream=0):
+    _check(lib().vit_op_layernorm(h, dtype, rows, cols, x, gain, shift, eps, y, stream), "vit_op_layernorm")
+
+
+def vit_op_linear(h, dtype, M, N, K, a, w, bias, epilogue, residual, out, stream=0):
+    _check(lib().vit_op_linear(h, dtype, M, N, K, a, w, bias, epilogue, residual, out, stream), "vit_op_linear")
+
+
+def vit_op_attention(h, dtype, images, T, heads, d, qkv, out, stream=0):
+    _check(lib().vit_op_attention(h, dtype, images, T, heads, d, qkv, out, stream), "vit_op_attention")
+
+
+# ---- convenience object: owns a handle and torch-allocated buffers --------------------------------
+class VitModel:
+    """A model instance plus torch-allocated workspaces.  All compute happens in the library."""
+
+    def __init__(self, shape, host_params: np.ndarray, dtype=VIT_BF16, max_microbatch=1, device="cuda:0"):
+        import torch
+        self.torch = torch
+        self.shape = shape
+        self.device = torch.device(device)
+        self.cfg = make_config(shape, dtype, max_microbatch)
+        self.act_dtype = torch.bfloat16 if dtype == VIT_BF16 else torch.float32
+        self.T = (shape.image_size // shape.patch_size) ** 2 + 1
+        with torch.cuda.device(self.device):
+            self.h = vit_create(self.cfg, host_params)
+        self._ws = {}
+
+    def close(self):
+        if getattr(self, "h", None):
+            with self.torch.cuda.device(self.device):
+                vit_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _stream(self, stream):
+        return (stream or self.torch.cuda.current_stream(self.device)).cuda_stream
+
+    def workspace(self, microbatch, key="default"):
+        n = vit_workspace_bytes(self.cfg, microbatch)
+        buf = self._ws.get(key)
+        if buf is None or buf.numel() < n:
+            buf = self.torch.empty(n, dtype=self.torch.uint8, device=self.device)
+            self._ws[key] = buf
+        return buf
+
+    def patch_embed(self, pixels, stream=None):
+        mb = pixels.shape[0]
+        assert pixels.dtype == self.torch.float32 and pixels.is_contiguous()
+        out = self.torch.empty((mb, self.T, self.shape.hidden), dtype=self.act_dtype, device=self.device)
+        ws = self.workspace(mb)
+        vit_patch_embed(self.h, mb, pixels.data_ptr(), out.data_ptr(), ws.data_ptr(), ws.numel(), self._stream(stream))
+        return out
+
+    def run_stage(self, layer_begin, layer_end, x, out=None, stream=None):
+        mb = x.shape[0]
+        assert x.dtype == self.act_dtype and x.is_contiguous()
+        if out is None:
+            out = self.torch.empty_like(x)
+        ws = self.workspace(mb)
+        vit_run_stage(self.h, layer_begin, layer_end, mb, x.data_ptr(), out.data_ptr(), ws.data_ptr(),
+                      ws.numel(), self._stream(stream))
+        return out
+
+    def head(self, x, stream=None):
+        mb = x.shape[0]
+        logits = self.torch.empty((mb, self.shape.num_classes), dtype=self.torch.float32, device=self.device)
+        ws = self.workspace(mb)
+        vit_head(self.h, mb, x.data_ptr(), logits.data_ptr(), ws.data_ptr(), ws.numel(), self._stream(stream))
+        return logits
+
+    def forward(self, pixels, stages=None):
+        stages = stages or [(0, self.shape.layers)]
+        x = self.patch_embed(pixels)
+        for lb, le in stages:
+            x = self.run_stage(lb, le, x, out=x)
+        return self.head(x)
+
+    def make_pipeline_buffers(self, microbatch, n_streams):
+        n = vit_pipeline_workspace_bytes(self.cfg, microbatch)
+        wss = [self.torch.empty(n, dtype=self.torch.uint8, device=self.device) for _ in range(n_streams)]
+        streams = [self.torch.cuda.Stream(self.device) for _ in range(n_streams)]
+        return wss, streams, n
+
+    def run_pipeline(self, stage_layers, microbatch, pixels, logits, wss, streams, ws_bytes, host=False):
+        batch = pixels.shape[0]
+        fn = vit_run_pipeline_host if host else vit_run_pipeline
+        fn(self.h, list(stage_layers), batch, microbatch, pixels.data_ptr(), logits.data_ptr(),
+           [w.data_ptr() for w in wss], ws_bytes, [s.cuda_stream for s in streams])
+
+    def check(self, stream=None):
+        vit_check_status(self.h, self._stream(stream))
+
+    @property
+    def launches(self):
+        return vit_launch_count(self.h)

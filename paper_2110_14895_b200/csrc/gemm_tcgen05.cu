@@ -1,0 +1,442 @@
+// Linear layers on the 5th-generation tensor cores:  out[M,N] = epi(a[M,K] . w[N,K]^T + bias).
+//
+// Persistent, warp-specialised kernel, one CTA per SM:
+//   warp 0      TMA producer: 128 x 64 tile of a and BN x 64 tile of w per stage, 128-byte swizzle
+//   warp 1      allocates tensor memory and issues tcgen05.mma (128 x BN x 16 per instruction)
+//   warps 2..9  epilogue: tcgen05.ld the fp32 accumulator, bias / GELU / residual, bf16 stores
+// Two accumulators live in tensor memory (2 x BN columns) so the epilogue of tile i overlaps the
+// main loop of tile i+1.  Tiles are handed out statically (tile = blockIdx.x + i * gridDim.x).
+// Every mbarrier wait is bounded; on expiry the CTA raises the device status word and leaves.
+#include "vit_internal.h"
+
+#include <cuda.h>
+
+namespace vit {
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;        // 64 bf16 = 128 bytes = one swizzle row
+constexpr int UMMA_K = 16;
+constexpr int NUM_EPI_WARPS = 8;
+constexpr int NUM_THREADS = (2 + NUM_EPI_WARPS) * 32;
+constexpr long long WAIT_LIMIT_CYCLES = 1ll << 31;
+
+template <int BN> struct Cfg {
+  static constexpr int STAGES = (BN == 256) ? 4 : 6;
+  static constexpr int A_BYTES = BM * BK * 2;
+  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int TMEM_COLS = 2 * BN;                 // 512 or 256: a power of two
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false if the wait expired or another thread of the CTA gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+      *abort_flag = 1;
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(tm)), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes, groups
+// of 8 rows 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);        // start address
+  d |= (uint64_t)1 << 16;                          // leading-dimension byte offset (unused with swizzle)
+  d |= (uint64_t)(1024 >> 4) << 32;                // stride-dimension byte offset: 8 rows x 128 B
+  d |= (uint64_t)1 << 46;                          // descriptor version for this architecture
+  d |= (uint64_t)2 << 61;                          // swizzle mode: 128 bytes
+  return d;
+}
+
+// Instruction descriptor for kind::f16: fp32 accumulate, bf16 x bf16, both operands K-major.
+template <int BN> __host__ __device__ constexpr uint32_t make_idesc() {
+  return (1u << 4)                       // D format: f32
+         | (1u << 7)                     // A format: bf16
+         | (1u << 10)                    // B format: bf16
+         | ((uint32_t)(BN >> 3) << 17)   // N / 8
+         | ((uint32_t)(BM >> 4) << 24);  // M / 16
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc,
+                                          uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+      "}\n" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+        "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]),
+        "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ float gelu_erf(float v) {
+  return 0.5f * v * (1.0f + erff(v * 0.70710678118654752440f));
+}
+
+struct TcParams {
+  int M, N, K;
+  const float* bias;
+  const bf16* residual;   // EPI_BIAS_RESIDUAL
+  const float* pos;       // EPI_BIAS_POS
+  int n_patches;
+  bf16* out;
+  int ldo;
+  int tiles_m, tiles_n;
+  int* dev_status;
+};
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w,
+                 const TcParams p) {
+  using C = Cfg<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  // 1024-byte alignment: the swizzle pattern and the descriptors assume it
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* tiles = smem;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::STAGES * C::STAGE_BYTES);
+  uint64_t* full_bar = bars;                       // [STAGES]
+  uint64_t* empty_bar = bars + C::STAGES;          // [STAGES]
+  uint64_t* tfull_bar = bars + 2 * C::STAGES;      // [2]
+  uint64_t* tempty_bar = bars + 2 * C::STAGES + 2; // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * C::STAGES + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int num_kb = (p.K + BK - 1) / BK;
+  const int total_tiles = p.tiles_m * p.tiles_n;
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int i = 0; i < C::STAGES; ++i) {
+      mbar_init(smem_u32(&full_bar[i]), 1);
+      mbar_init(smem_u32(&empty_bar[i]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&tfull_bar[i]), 1);
+      mbar_init(smem_u32(&tempty_bar[i]), NUM_EPI_WARPS);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_a)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_w)) : "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(tmem_slot)),
+                 "r"((uint32_t)C::TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int m0 = (tile / p.tiles_n) * BM, n0 = (tile % p.tiles_n) * BN;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1, abort_flag)) { ok = false; break; }
+          const uint32_t fb = smem_u32(&full_bar[stage]);
+          mbar_arrive_expect_tx(fb, C::STAGE_BYTES);
+          const uint32_t sa = smem_u32(tiles + stage * C::STAGE_BYTES);
+          tma_load_2d(sa, &tm_a, kb * BK, m0, fb);
+          tma_load_2d(sa + C::A_BYTES, &tm_w, kb * BK, n0, fb);
+          if (++stage == C::STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc<BN>();
+      int stage = 0;
+      uint32_t phase = 0;
+      int buf = 0;
+      uint32_t aphase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        if (!mbar_wait(smem_u32(&tempty_bar[buf]), aphase ^ 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!mbar_wait(smem_u32(&full_bar[stage]), phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(tiles + stage * C::STAGE_BYTES);
+          const uint64_t adesc = make_smem_desc(sa);
+          const uint64_t bdesc = make_smem_desc(sa + C::A_BYTES);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            // advancing 16 elements along K = 32 bytes = 2 units of the encoded start address
+            umma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
+                      (kb > 0 || k > 0) ? 1u : 0u);
+          }
+          umma_commit(smem_u32(&empty_bar[stage]));   // frees the stage when these MMAs retire
+          if (++stage == C::STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        umma_commit(smem_u32(&tfull_bar[buf]));       // accumulator complete
+        if (++buf == 2) { buf = 0; aphase ^= 1; }
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue
+    const int ew = warp - 2;
+    const int quarter = warp & 3;                 // tensor-memory lanes this warp may read
+    const int half = ew >> 2;                     // which half of the BN columns
+    constexpr int COLS_PER_WARP = BN / 2;
+    int buf = 0;
+    uint32_t aphase = 0;
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+      const int m0 = (tile / p.tiles_n) * BM, n0 = (tile % p.tiles_n) * BN;
+      if (!mbar_wait(smem_u32(&tfull_bar[buf]), aphase, abort_flag)) break;
+      tc_fence_after();
+      const int row = m0 + quarter * 32 + lane;
+      const bool row_ok = row < p.M;
+      size_t orow = (size_t)row;
+      const float* posrow = nullptr;
+      if (EPI == EPI_BIAS_POS) {
+        const int img = row / p.n_patches, pt = row - img * p.n_patches;
+        orow = (size_t)img * (p.n_patches + 1) + 1 + pt;
+        posrow = p.pos + (size_t)(1 + pt) * p.N;
+      }
+#pragma unroll 1
+      for (int ch = 0; ch < COLS_PER_WARP / 32; ++ch) {
+        const int cl = half * COLS_PER_WARP + ch * 32;   // column inside the tile
+        const int c0 = n0 + cl;
+        if (c0 >= p.N) break;                            // uniform across the warp
+        uint32_t r[32];
+        tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cl), r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          const int c = c0 + g * 8;
+          if (c >= p.N) break;
+          const float4 b0 = __ldg(reinterpret_cast<const float4*>(p.bias + c));
+          const float4 b1 = __ldg(reinterpret_cast<const float4*>(p.bias + c) + 1);
+          float v[8];
+          v[0] = __uint_as_float(r[g * 8 + 0]) + b0.x;
+          v[1] = __uint_as_float(r[g * 8 + 1]) + b0.y;
+          v[2] = __uint_as_float(r[g * 8 + 2]) + b0.z;
+          v[3] = __uint_as_float(r[g * 8 + 3]) + b0.w;
+          v[4] = __uint_as_float(r[g * 8 + 4]) + b1.x;
+          v[5] = __uint_as_float(r[g * 8 + 5]) + b1.y;
+          v[6] = __uint_as_float(r[g * 8 + 6]) + b1.z;
+          v[7] = __uint_as_float(r[g * 8 + 7]) + b1.w;
+          if (row_ok) {
+            if (EPI == EPI_BIAS_GELU) {
+#pragma unroll
+              for (int e = 0; e < 8; ++e) v[e] = gelu_erf(v[e]);
+            } else if (EPI == EPI_BIAS_RESIDUAL) {
+              const uint4 u = *reinterpret_cast<const uint4*>(p.residual + orow * p.ldo + c);
+              const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float2 f = __bfloat1622float2(h[e]);
+                v[2 * e] += f.x;
+                v[2 * e + 1] += f.y;
+              }
+            } else if (EPI == EPI_BIAS_POS) {
+              const float4 p0 = __ldg(reinterpret_cast<const float4*>(posrow + c));
+              const float4 p1 = __ldg(reinterpret_cast<const float4*>(posrow + c) + 1);
+              v[0] += p0.x; v[1] += p0.y; v[2] += p0.z; v[3] += p0.w;
+              v[4] += p1.x; v[5] += p1.y; v[6] += p1.z; v[7] += p1.w;
+            }
+            uint4 o;
+            __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) h[e] = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
+            *reinterpret_cast<uint4*>(p.out + orow * p.ldo + c) = o;
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[buf]));
+      if (++buf == 2) { buf = 0; aphase ^= 1; }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  __syncwarp();
+  if (*abort_flag) __nanosleep(200000);   // let copies and MMAs in flight land before leaving
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (threadIdx.x == 0 && *abort_flag) atomicExch(p.dev_status, (int)VIT_ERR_TIMEOUT);
+  if (warp == 1) {
+    __syncwarp();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                 "r"((uint32_t)C::TMEM_COLS)
+                 : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+int g_num_sms = 0;
+
+bool encode_2d_bf16(CUtensorMap* tm, const void* base, int rows, int cols, int ld, int box_rows) {
+  const cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t gstride[1] = {(cuuint64_t)ld * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride,
+                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN, int EPI>
+cudaError_t launch_variant(const CUtensorMap& ta, const CUtensorMap& tw, const TcParams& p,
+                           cudaStream_t s) {
+  static bool configured = false;   // benign race: the attribute is idempotent
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(linear_tc_kernel<BN, EPI>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         Cfg<BN>::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  const int total = p.tiles_m * p.tiles_n;
+  const int grid = total < g_num_sms ? total : g_num_sms;
+  linear_tc_kernel<BN, EPI><<<grid, NUM_THREADS, Cfg<BN>::SMEM_BYTES, s>>>(ta, tw, p);
+  return cudaGetLastError();
+}
+
+template <int BN>
+cudaError_t launch_bn(int epi, const CUtensorMap& ta, const CUtensorMap& tw, const TcParams& p,
+                      cudaStream_t s) {
+  switch (epi) {
+    case EPI_BIAS: return launch_variant<BN, EPI_BIAS>(ta, tw, p, s);
+    case EPI_BIAS_GELU: return launch_variant<BN, EPI_BIAS_GELU>(ta, tw, p, s);
+    case EPI_BIAS_RESIDUAL: return launch_variant<BN, EPI_BIAS_RESIDUAL>(ta, tw, p, s);
+    case EPI_BIAS_POS: return launch_variant<BN, EPI_BIAS_POS>(ta, tw, p, s);
+  }
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace
+
+bool tc_gemm_init() {
+  if (g_encode) return true;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+      q != cudaDriverEntryPointSuccess || fn == nullptr)
+    return false;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  if (cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
+  g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  return true;
+}
+
+cudaError_t launch_linear_tc(const LinearArgs& a, int* dev_status, cudaStream_t s) {
+  if (a.M <= 0 || a.N <= 0) return cudaSuccess;
+  if (!g_encode) return cudaErrorNotReady;
+  if (a.K % 8 || a.N % 8 || a.lda % 8 || a.ldw % 8 || a.ldo % 8 || a.K <= 0) return cudaErrorInvalidValue;
+  if ((reinterpret_cast<uintptr_t>(a.a) | reinterpret_cast<uintptr_t>(a.w) |
+       reinterpret_cast<uintptr_t>(a.out) | reinterpret_cast<uintptr_t>(a.residual)) & 15)
+    return cudaErrorInvalidValue;
+  const int tiles_m = (a.M + BM - 1) / BM;
+  // a full wave of 128x256 tiles, else the narrower tile to fill more SMs; shape-only decision
+  const bool wide = (long long)tiles_m * ((a.N + 255) / 256) >= g_num_sms;
+  const int bn = wide ? 256 : 128;
+  TcParams p;
+  p.M = a.M; p.N = a.N; p.K = a.K;
+  p.bias = a.bias;
+  p.residual = static_cast<const bf16*>(a.residual);
+  p.pos = a.pos;
+  p.n_patches = a.n_patches > 0 ? a.n_patches : 1;
+  p.out = static_cast<bf16*>(a.out);
+  p.ldo = a.ldo;
+  p.tiles_m = tiles_m;
+  p.tiles_n = (a.N + bn - 1) / bn;
+  p.dev_status = dev_status;
+  CUtensorMap ta, tw;
+  if (!encode_2d_bf16(&ta, a.a, a.M, a.K, a.lda, BM)) return cudaErrorInvalidValue;
+  if (!encode_2d_bf16(&tw, a.w, a.N, a.K, a.ldw, bn)) return cudaErrorInvalidValue;
+  return wide ? launch_bn<256>(a.epilogue, ta, tw, p, s) : launch_bn<128>(a.epilogue, ta, tw, p, s);
+}
+
+}  // namespace vit

@@ -1,0 +1,83 @@
+// Internal declarations shared by the library's translation units (not part of the C boundary).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+#include <atomic>
+
+#include "../../include/vit.h"
+
+namespace vit {
+
+typedef __nv_bfloat16 bf16;
+
+// Epilogue selector of the linear kernels.
+enum Epilogue : int {
+  EPI_BIAS = 0,          // out = acc + bias
+  EPI_BIAS_GELU = 1,     // out = gelu(acc + bias), erf form
+  EPI_BIAS_RESIDUAL = 2, // out = acc + bias + residual[row, col]
+  EPI_BIAS_POS = 3       // patch embed: row r of the GEMM is patch r % n_patches of image r / n_patches;
+                         // out[image*T + 1 + patch, col] = acc + bias + pos[1 + patch, col]
+};
+
+struct LinearArgs {
+  int M, N, K;            // out[M,N] = a[M,K] . w[N,K]^T
+  const void* a;          // activation type, row stride lda elements
+  int lda;
+  const void* w;          // activation type, row stride K... (ldw elements)
+  int ldw;
+  const float* bias;      // [N]
+  int epilogue;
+  const void* residual;   // EPI_BIAS_RESIDUAL: [M, N] stride ldo; may alias out
+  const float* pos;       // EPI_BIAS_POS: [T, N] fp32
+  int n_patches;          // EPI_BIAS_POS
+  void* out;              // activation type, row stride ldo
+  int ldo;
+};
+
+struct LayerWeights {
+  const float *ln1_g, *ln1_b, *bqkv, *bo, *ln2_g, *ln2_b, *b1, *b2;
+  const void *Wqkv, *Wo, *W1, *W2;   // activation type, [out, in]
+};
+
+struct Handle {
+  vit_config cfg;
+  int T, n_patches, d, patch_k, patch_k_pad;
+  size_t act_bytes;                  // bytes of one activation element
+  void* dev_blob;                    // every parameter, one allocation
+  size_t dev_blob_bytes;
+  const void* patch_W;               // [H, patch_k_pad]
+  const float *patch_b, *cls, *pos;
+  LayerWeights* layers;              // host array [L]
+  const float *lnf_g, *lnf_b, *head_b;
+  const void* head_W;                // [classes, H]
+  int* dev_status;                   // device status word (0 = ok)
+  std::atomic<uint64_t> launches;
+};
+
+// ---- kernel launchers (each returns a cudaError_t from the launch) ------------------------
+// bf16 family
+cudaError_t launch_layernorm_bf16(const bf16* x, const float* g, const float* b, float eps,
+                                  bf16* y, int rows, int cols, cudaStream_t s);
+cudaError_t launch_linear_tc(const LinearArgs& a, int* dev_status, cudaStream_t s);   // tcgen05 GEMM
+cudaError_t launch_attention_bf16(const bf16* qkv, bf16* out, int images, int T, int heads, int d,
+                                  cudaStream_t s);
+// fp32 family (SIMT)
+cudaError_t launch_layernorm_f32(const float* x, const float* g, const float* b, float eps,
+                                 float* y, int rows, int cols, cudaStream_t s);
+cudaError_t launch_linear_f32(const LinearArgs& a, cudaStream_t s);
+cudaError_t launch_attention_f32(const float* qkv, float* out, int images, int T, int heads, int d,
+                                 cudaStream_t s);
+// book-ends, both families (act_bf16 selects the element type)
+cudaError_t launch_im2col(const float* pixels, void* cols, int images, int C, int S, int P,
+                          int k_pad, bool act_bf16, cudaStream_t s);
+cudaError_t launch_cls_rows(const float* cls, const float* pos, void* tokens, int images, int T,
+                            int H, bool act_bf16, cudaStream_t s);
+cudaError_t launch_head(const void* tokens, const float* g, const float* b, float eps,
+                        const void* W, const float* bias, float* feat_scratch, float* logits,
+                        int images, int T, int H, int classes, bool act_bf16, cudaStream_t s);
+
+bool tc_gemm_init();   // resolves the driver's tensor-map encoder; false if unavailable
+
+}  // namespace vit

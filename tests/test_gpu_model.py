@@ -1,0 +1,220 @@
+"""End-to-end parity of the CUDA path with the CPU oracle on the same seeded inputs, and the
+stage-composition invariant on the GPU.  Everything goes through the C boundary."""
+import numpy as np
+import pytest
+
+import vitgen
+from oracle import vit_oracle as O
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+def _vit():
+    import paper_2110_14895_b200 as vit
+    return vit
+
+
+def logits_within_tolerance(got, want, rel_max, min_cos=None):
+    """max |dlogit| <= rel_max * max |logit| over the whole array; cosine per image."""
+    got = np.asarray(got, dtype=np.float64)
+    scale = np.abs(want).max()
+    err = np.abs(got - want).max()
+    cos = (got * want).sum(-1) / (np.linalg.norm(got, axis=-1) * np.linalg.norm(want, axis=-1))
+    ok = err <= rel_max * scale and (min_cos is None or cos.min() >= min_cos)
+    return ok, f"max|d|={err:.3e} ({err / scale:.3e} of max|logit|), min cos={cos.min():.6f}"
+
+
+def _model(shape, dtype, max_mb, seed=0, bf16_weights=True, ln_affine=False):
+    vit = _vit()
+    params, blob = vitgen.make_params(shape, seed=seed, bf16=bf16_weights, ln_affine=ln_affine)
+    return vit, vit.VitModel(shape, blob, dtype, max_mb), params
+
+
+# ---------------------------------------------------------------------------------------------
+# ViT-Tiny/16, batch 1, fp32 mode, two stages [0,6)+[6,12): within 1e-3 of the oracle.
+def test_tiny_fp32_two_stages_matches_oracle():
+    shape = vitgen.preset("tiny16")
+    vit, m, params = _model(shape, _vit().VIT_FP32, 2, bf16_weights=False)
+    pix = vitgen.make_pixels(shape, 1, seed=0)
+    got = m.forward(torch.from_numpy(pix).cuda(), stages=[(0, 6), (6, 12)])
+    m.check()
+    want = O.forward(params, shape, pix, [(0, 6), (6, 12)])
+    ok, msg = logits_within_tolerance(got.cpu().numpy(), want, 1e-3)
+    assert ok, msg
+    m.close()
+
+
+@pytest.mark.parametrize("dtype_name", ["bf16", "fp32"])
+def test_tiny_intermediate_tensors_match_oracle(dtype_name):
+    vit = _vit()
+    dtype = vit.VIT_BF16 if dtype_name == "bf16" else vit.VIT_FP32
+    shape = vitgen.preset("tiny16").with_(layers=2)
+    vit, m, params = _model(shape, dtype, 3, seed=5, ln_affine=True)
+    pix = vitgen.make_pixels(shape, 3, seed=5)
+    x = m.patch_embed(torch.from_numpy(pix).cuda())
+    m.check()
+    want = O.patch_embed(params, shape, pix)
+    tol = 1e-5 if dtype_name == "fp32" else 2.0 ** -8
+    got = x.float().cpu().numpy()
+    assert np.abs(got - want).max() <= tol * np.abs(want).max() + (3e-3 if dtype_name == "bf16" else 0)
+    y = m.run_stage(0, 2, x)
+    m.check()
+    want2 = O.run_stage(params, shape, 0, 2, want)
+    rel = np.abs(y.float().cpu().numpy() - want2).max() / np.abs(want2).max()
+    assert rel <= (1e-4 if dtype_name == "fp32" else 2e-2), rel
+    m.close()
+
+
+def test_tiny_bf16_matches_oracle_and_composes_bit_exactly():
+    shape = vitgen.preset("tiny16")
+    vit, m, params = _model(shape, _vit().VIT_BF16, 4)
+    pix = vitgen.make_pixels(shape, 4, seed=0)
+    dpix = torch.from_numpy(pix).cuda()
+    whole = m.forward(dpix)
+    want = O.forward(params, shape, pix)
+    ok, msg = logits_within_tolerance(whole.cpu().numpy(), want, 2e-2, 0.9995)
+    assert ok, msg
+    x0 = m.patch_embed(dpix)
+    ref = m.run_stage(0, shape.layers, x0)
+    for k in range(1, shape.layers):
+        a = m.run_stage(0, k, x0)
+        b = m.run_stage(k, shape.layers, a, out=a)       # second stage in place
+        assert torch.equal(ref, b), k
+    m.check()
+    m.close()
+
+
+def test_stage_argument_errors():
+    shape = vitgen.preset("tiny16").with_(layers=3)
+    vit, m, _ = _model(shape, _vit().VIT_BF16, 2)
+    x = torch.zeros((2, m.T, shape.hidden), dtype=torch.bfloat16, device="cuda")
+    ws = m.workspace(2)
+    def run(lb, le, mb=2, inp=None, out=None, wsb=None):
+        vit.vit_run_stage(m.h, lb, le, mb, (inp or x.data_ptr()), (out or x.data_ptr()), ws.data_ptr(),
+                          ws.numel() if wsb is None else wsb)
+    for lb, le in [(0, 0), (2, 1), (-1, 2), (0, 4), (3, 3)]:
+        with pytest.raises(vit.VitError) as e:
+            run(lb, le)
+        assert e.value.status == vit.VIT_ERR_RANGE
+    with pytest.raises(vit.VitError) as e:
+        run(0, 1, mb=3)
+    assert e.value.status == vit.VIT_ERR_INVALID_ARG
+    with pytest.raises(vit.VitError) as e:
+        run(0, 1, wsb=1024)
+    assert e.value.status == vit.VIT_ERR_WORKSPACE
+    with pytest.raises(vit.VitError) as e:
+        run(0, 1, out=x.data_ptr() + 256)            # partial overlap
+    assert e.value.status == vit.VIT_ERR_INVALID_ARG
+    before = m.launches
+    with pytest.raises(vit.VitError):
+        run(0, 9)
+    assert m.launches == before                       # a failed call launches nothing
+    m.close()
+
+
+# ---------------------------------------------------------------------------------------------
+def _pipeline_vs_oracle(name, batch, mb, stages, n_streams, sample, host=False):
+    """Runs the stage runner on the full batch; the oracle evaluates the sampled images only
+    (images are independent, so that is the same function)."""
+    shape = vitgen.preset(name)
+    vit, m, params = _model(shape, _vit().VIT_BF16, mb)
+    pix = vitgen.make_pixels(shape, batch, seed=0)
+    wss, streams, wsb = m.make_pipeline_buffers(mb, n_streams)
+    counts = [le - lb for lb, le in stages]
+    if host:
+        hp = torch.from_numpy(pix).pin_memory()
+        logits = torch.empty((batch, shape.num_classes), dtype=torch.float32).pin_memory()
+        torch.cuda.synchronize()
+        m.run_pipeline(counts, mb, hp, logits, wss, streams, wsb, host=True)
+    else:
+        dp = torch.from_numpy(pix).cuda()
+        logits = torch.full((batch, shape.num_classes), float("nan"), dtype=torch.float32, device="cuda")
+        torch.cuda.synchronize()
+        m.run_pipeline(counts, mb, dp, logits, wss, streams, wsb)
+    for s in streams:
+        m.check(s)
+    got = logits.cpu().numpy()
+    assert np.isfinite(got).all()
+    want = O.forward(params, shape, pix[sample])
+    ok, msg = logits_within_tolerance(got[sample], want, 2e-2, 0.9995)
+    assert ok, msg
+    return vit, m, pix, got
+
+
+def test_base16_batch64_four_microbatches_four_stages():
+    sample = [0, 15, 16, 31, 47, 48, 62, 63]
+    vit, m, pix, got = _pipeline_vs_oracle("base16", 64, 16, vitgen.equal_partition(4, 12), 4, sample)
+    # the single-call result on one microbatch is bit-identical to the staged pipeline result
+    one = m.forward(torch.from_numpy(pix[16:32]).cuda())
+    assert np.array_equal(one.cpu().numpy(), got[16:32])
+    m.close()
+
+
+def test_base16_host_buffers_pipeline():
+    _, m, _, _ = _pipeline_vs_oracle("base16", 8, 4, vitgen.equal_partition(4, 12), 2, [0, 3, 4, 7], host=True)
+    m.close()
+
+
+def test_large16_batch128_microbatch8_uneven_16_stages():
+    stages = vitgen.uneven_partition(16, 24, seed=0)
+    sample = [0, 7, 8, 64, 71, 120, 127]
+    vit, m, pix, got = _pipeline_vs_oracle("large16", 128, 8, stages, 1, sample)
+    one = m.forward(torch.from_numpy(pix[64:72]).cuda())
+    assert np.array_equal(one.cpu().numpy(), got[64:72])
+    m.close()
+
+
+def test_huge14_batch128_single_stage_equals_eight_stages_and_oracle():
+    shape = vitgen.preset("huge14")
+    vit, m, params = _model(shape, _vit().VIT_BF16, 128)
+    B = 128
+    pix = vitgen.make_pixels(shape, B, seed=0)
+    dp = torch.from_numpy(pix).cuda()
+    x0 = m.patch_embed(dp)
+    a = m.run_stage(0, 32, x0)
+    la = m.head(a)
+    b = x0.clone()
+    for lb, le in vitgen.equal_partition(8, 32):
+        m.run_stage(lb, le, b, out=b)
+    lb_ = m.head(b)
+    m.check()
+    assert torch.equal(a, b)
+    assert torch.equal(la, lb_)
+    sample = [0, 1, 63, 64, 100, 127]
+    want = O.forward(params, shape, pix[sample])
+    ok, msg = logits_within_tolerance(la.cpu().numpy()[sample], want, 2e-2, 0.9995)
+    assert ok, msg
+    m.close()
+
+
+def test_huge14_microbatch_sweep_on_streams_is_consistent():
+    """Microbatch sizes through a 4-stage partition on streams: every size gives finite logits
+    that agree with the batch-of-one result within the bf16 tolerance (tile shapes may differ
+    between sizes, so bit equality is not required)."""
+    shape = vitgen.preset("huge14")
+    vit, m, params = _model(shape, _vit().VIT_BF16, 32)
+    B = 32
+    pix = vitgen.make_pixels(shape, B, seed=0)
+    dp = torch.from_numpy(pix).cuda()
+    ref = None
+    for mb in (1, 2, 4, 8, 16, 32):
+        ns = min(4, B // mb)
+        wss, streams, wsb = m.make_pipeline_buffers(mb, ns)
+        logits = torch.full((B, shape.num_classes), float("nan"), dtype=torch.float32, device="cuda")
+        torch.cuda.synchronize()
+        m.run_pipeline([8, 8, 8, 8], mb, dp, logits, wss, streams, wsb)
+        for s in streams:
+            m.check(s)
+        got = logits.cpu().numpy()
+        assert np.isfinite(got).all()
+        if ref is None:
+            ref = got
+            want = O.forward(params, shape, pix[[0, 31]])
+            ok, msg = logits_within_tolerance(got[[0, 31]], want, 2e-2, 0.9995)
+            assert ok, msg
+        else:
+            ok, msg = logits_within_tolerance(got, ref.astype(np.float64), 2e-2, 0.9995)
+            assert ok, (mb, msg)
+        del wss
+    m.close()

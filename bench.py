@@ -1,0 +1,323 @@
+#!/usr/bin/env python
+"""Benchmark of the ViT pipeline-stage forward on B200.
+
+One step = one pass of the whole hot path over one batch of synthetic images: patch embed,
+every stage of the partition, classification head.  Prints ONE JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload huge14|large16|base16]
+  python bench.py --impl reference ...     # times the CPU oracle instead (bounded sample per step)
+
+With N > 1 (launched under torchrun) every rank runs an independent replica on its own GPU
+(images are independent, there is no data-path collective); the value is the aggregate.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import vitgen  # noqa: E402
+
+WORKLOADS = {
+    # name: (preset, batch, microbatch, stages) -- the single-GPU configurations of the metric
+    "huge14": ("huge14", 128, 128, 1),
+    "large16": ("large16", 128, 8, 16),
+    "base16": ("base16", 64, 16, 4),
+}
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def flops_per_image(s):
+    T, H, F = s.tokens, s.hidden, s.mlp_dim
+    gemm = {
+        "qkv": 2 * T * 3 * H * H, "outproj": 2 * T * H * H, "fc1": 2 * T * H * F, "fc2": 2 * T * H * F,
+    }
+    attn = 4 * T * T * H
+    embed = 2 * s.n_patches * s.patch_k * H
+    head = 2 * H * s.num_classes
+    total = s.layers * (sum(gemm.values()) + attn) + embed + head
+    return total, gemm, attn, embed
+
+
+def stage_counts(shape, n_stages, seed=0):
+    if n_stages == 1:
+        return [shape.layers]
+    if shape.layers % n_stages == 0 and n_stages != 16:
+        return [shape.layers // n_stages] * n_stages
+    return [b - a for a, b in vitgen.uneven_partition(n_stages, shape.layers, seed)]
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
+    return dict(FALLBACK_PEAKS) | {"source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.lines, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=lambda: self.lines.extend(self.proc.stdout), daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def __exit__(self, *a):
+        if self.proc:
+            time.sleep(0.15)
+            self.proc.terminate()
+            self.t.join(timeout=2)
+
+    def summary(self):
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); pw.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": max(mx), "power_w": float(np.median(pw)),
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_images_per_s(shape, n_images, seed=0, params=None):
+    """Times the CPU oracle, as it stands, on `n_images` images of the workload."""
+    from oracle import vit_oracle as O
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([i.get("num_threads", 1) for i in threadpool_info()] or [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    if params is None:
+        params, _ = vitgen.make_params(shape, seed=seed)
+    pix = vitgen.make_pixels(shape, n_images, seed=seed)
+    t0 = time.perf_counter()
+    O.forward(params, shape, pix)
+    dt = time.perf_counter() - t0
+    return n_images / dt, cores, dt
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    preset, batch, mb, n_stages = WORKLOADS[args.workload]
+    shape = vitgen.preset(preset)
+    params, _ = vitgen.make_params(shape, seed=0)
+    per_step = 1
+    times = []
+    cores = 1
+    for i in range(args.warmup + args.steps):
+        ips, cores, dt = oracle_images_per_s(shape, per_step, params=params)
+        if i >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * float(np.mean(times))
+    value = per_step / (ms / 1e3)
+    line = {
+        "impl": "reference", "metric": "images/sec", "value": value, "unit": "images/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"ViT-{preset} forward, {shape.tokens} tokens, {shape.layers} layers",
+                   "images_per_step": per_step},
+        "cpu_baseline": {"value": value, "unit": "images/s", "cores": cores, "kind": "oracle",
+                         "sample": f"{per_step} image per step of the {preset} workload, numpy fp64"},
+        "e2e": {"value": value, "unit": "images/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--workload", default="huge14", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2110_14895_b200 as vit
+
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    preset, batch, mb, n_stages = WORKLOADS[args.workload]
+    shape = vitgen.preset(preset)
+    counts = stage_counts(shape, n_stages)
+    _, blob = vitgen.make_params(shape, seed=0)
+    model = vit.VitModel(shape, blob, vit.VIT_BF16, mb, device=dev)
+    del blob
+    pix_host = torch.from_numpy(vitgen.make_pixels(shape, batch, seed=rank)).pin_memory()
+    pix = pix_host.to(dev)
+    logits = torch.empty((batch, shape.num_classes), dtype=torch.float32, device=dev)
+    n_streams = 1
+    wss, streams, wsb = model.make_pipeline_buffers(mb, n_streams)
+
+    def step():
+        model.run_pipeline(counts, mb, pix, logits, wss, streams, wsb)
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def timed(fn, steps, stream_list):
+        barrier()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(stream_list[0])
+        for s in stream_list[1:]:
+            s.wait_event(ev0)
+        for _ in range(steps):
+            fn()
+        for s in stream_list[1:]:
+            e = torch.cuda.Event()
+            e.record(s)
+            stream_list[0].wait_event(e)
+        ev1.record(stream_list[0])
+        barrier()
+        ms = ev0.elapsed_time(ev1)
+        if world > 1:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    for _ in range(args.warmup):
+        step()
+    model.check(streams[0])
+
+    launches0 = model.launches
+    with ClockSampler(local) as clk:
+        ms_total = timed(step, args.steps, streams)
+    launches = model.launches - launches0
+    model.check(streams[0])
+    ms_step = ms_total / args.steps
+    value = world * batch / (ms_step / 1e3)
+
+    # per-kernel timing over the same steps (event pairs around every launch, same stream)
+    vit.vit_profile_enable(model.h, True)
+    prof_steps = min(args.steps, 5)
+    timed(step, prof_steps, streams)
+    prof = vit.vit_profile_collect(model.h)
+    vit.vit_profile_enable(model.h, False)
+
+    # end to end: host pixels in, host logits out, through the host-buffer entry point
+    e2e_mb = min(mb, 32)
+    e2e_streams_n = min(4, max(1, batch // e2e_mb))
+    e_wss, e_streams, e_wsb = model.make_pipeline_buffers(e2e_mb, e2e_streams_n)
+    logits_host = torch.empty((batch, shape.num_classes), dtype=torch.float32).pin_memory()
+
+    def step_host():
+        model.run_pipeline(counts, e2e_mb, pix_host, logits_host, e_wss, e_streams, e_wsb, host=True)
+
+    for _ in range(2):
+        step_host()
+    e2e_steps = max(3, min(args.steps, 10))
+    ms_e2e = timed(step_host, e2e_steps, e_streams) / e2e_steps
+    for s in e_streams:
+        model.check(s)
+    e2e_value = world * batch / (ms_e2e / 1e3)
+
+    if rank == 0:
+        pk = peaks()
+        total_flops, gemm, attn, embed = flops_per_image(shape)
+        gemm_ms = sum(prof[k][0] for k in ("qkv", "outproj", "fc1", "fc2"))
+        gemm_launches = sum(prof[k][1] for k in ("qkv", "outproj", "fc1", "fc2"))
+        gemm_flops = sum(gemm.values()) * shape.layers * batch * prof_steps
+        achieved = gemm_flops / (gemm_ms / 1e3) / 1e12 if gemm_ms > 0 else None
+        peak = pk["bf16_tflops_sustained"]
+        per_class = {}
+        M = batch * shape.tokens
+        for k, (ms, n) in prof.items():
+            if n == 0:
+                continue
+            per_class[k] = {"ms_per_step": ms / prof_steps, "launches_per_step": n // prof_steps}
+            if k in gemm:
+                per_class[k]["tflops"] = gemm[k] * shape.layers * batch * prof_steps / (ms / 1e3) / 1e12
+            if k == "attention":
+                per_class[k]["tflops"] = attn * shape.layers * batch * prof_steps / (ms / 1e3) / 1e12
+            if k == "layernorm":
+                per_class[k]["gbs"] = 2 * shape.layers * prof_steps * (2 * M * shape.hidden * 2) / (ms / 1e3) / 1e9
+        line = {
+            "metric": "images/sec", "value": value, "unit": "images/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {
+                "workload": f"ViT-{preset} forward, batch {batch}, microbatch {mb}, stages {counts}, "
+                            f"{shape.tokens} tokens, {shape.layers} layers, hidden {shape.hidden}",
+                "global_batch": world * batch, "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                "l2": "activations and weights per layer exceed L2 (no flush needed)",
+            },
+            "tflops": value * total_flops / 1e12,
+            "frac_of_bf16_peak": {"burst": value * total_flops / 1e12 / world / pk["bf16_tflops"],
+                                  "sustained": value * total_flops / 1e12 / world / pk["bf16_tflops_sustained"],
+                                  "peaks": pk["source"]},
+            "e2e": {"value": e2e_value, "unit": "images/s",
+                    "h2d_bytes_per_step": int(pix_host.numel() * 4), "d2h_bytes_per_step": int(logits_host.numel() * 4),
+                    "microbatch": e2e_mb, "streams": e2e_streams_n},
+            "gpu_launches": int(launches),
+            "clocks": clk.summary(),
+            "roofline": {
+                "kernel": "linear_tc_kernel (QKV, out-proj, fc1, fc2 GEMMs)", "bound": "tensor",
+                "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak if achieved else None,
+                "peak_kind": f"{pk['source']} sustained bf16 (kernel timed inside a long step)",
+                "frac_of_burst": achieved / pk["bf16_tflops"] if achieved else None,
+                "launches": gemm_launches, "traffic": None,
+            },
+            "kernels": per_class,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            n_img = 2 if preset == "huge14" else 4
+            ips, cores, dt = oracle_images_per_s(shape, n_img)
+            line["cpu_baseline"] = {"value": ips, "unit": "images/s", "cores": cores, "kind": "oracle",
+                                    "sample": f"{n_img} images of the same workload, numpy fp64, {dt:.1f} s"}
+        print(json.dumps(line), flush=True)
+    model.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -149,6 +149,18 @@ uint64_t vit_launch_count(const vit_handle* h);
 
 const char* vit_status_string(int status);
 
+/* Per-kernel timing.  While enabled, every kernel launch of this handle is bracketed by a pair
+ * of CUDA events on the stream it is launched on.  vit_profile_collect synchronises the device,
+ * adds the elapsed milliseconds and launch counts per class into the two arrays of
+ * VIT_PROF_CLASSES entries, and clears the records.  Use from one host thread only. */
+enum {
+  VIT_PROF_LAYERNORM = 0, VIT_PROF_QKV = 1, VIT_PROF_ATTENTION = 2, VIT_PROF_OUTPROJ = 3,
+  VIT_PROF_FC1 = 4, VIT_PROF_FC2 = 5, VIT_PROF_EMBED = 6, VIT_PROF_HEAD = 7, VIT_PROF_OP = 8,
+  VIT_PROF_CLASSES = 9
+};
+int vit_profile_enable(vit_handle* h, int on);
+int vit_profile_collect(vit_handle* h, double* ms_by_class, uint64_t* launches_by_class);
+
 /* ---- single operations, exposed so that each kernel can be checked on its own ------------
  * All pointers dev; `dtype` selects the bf16 or fp32 kernel family as in vit_config.
  * They need a handle only for the device status word and the launch counter. */

@@ -24,8 +24,10 @@ EXPORTS = [
     "vit_param_count", "vit_workspace_bytes", "vit_pipeline_workspace_bytes", "vit_create",
     "vit_destroy", "vit_patch_embed", "vit_run_stage", "vit_head", "vit_run_pipeline",
     "vit_run_pipeline_host", "vit_check_status", "vit_launch_count", "vit_status_string",
-    "vit_op_layernorm", "vit_op_linear", "vit_op_attention",
+    "vit_op_layernorm", "vit_op_linear", "vit_op_attention", "vit_profile_enable",
+    "vit_profile_collect",
 ]
+PROF_CLASSES = ["layernorm", "qkv", "attention", "outproj", "fc1", "fc2", "embed", "head", "op"]
 
 
 class VitConfig(Structure):
@@ -87,6 +89,10 @@ def lib():
     L.vit_op_linear.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p]
     L.vit_op_attention.restype = c_int
     L.vit_op_attention.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p]
+    L.vit_profile_enable.restype = c_int
+    L.vit_profile_enable.argtypes = [c_void_p, c_int]
+    L.vit_profile_collect.restype = c_int
+    L.vit_profile_collect.argtypes = [c_void_p, P(ctypes.c_double), P(c_uint64)]
     _lib = L
     return L
 
@@ -174,6 +180,19 @@ def vit_check_status(h, stream=0) -> None:
 
 def vit_launch_count(h) -> int:
     return lib().vit_launch_count(h)
+
+
+def vit_profile_enable(h, on: bool) -> None:
+    _check(lib().vit_profile_enable(h, 1 if on else 0), "vit_profile_enable")
+
+
+def vit_profile_collect(h) -> dict:
+    """{class name: (milliseconds, launches)} since profiling was enabled or last collected."""
+    n = len(PROF_CLASSES)
+    ms = (ctypes.c_double * n)()
+    cnt = (c_uint64 * n)()
+    _check(lib().vit_profile_collect(h, ms, cnt), "vit_profile_collect")
+    return {PROF_CLASSES[i]: (ms[i], int(cnt[i])) for i in range(n)}
 
 
 def vit_op_layernorm(h, dtype, rows, cols, x, gain, shift, eps, y, stream=0):

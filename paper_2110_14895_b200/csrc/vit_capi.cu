@@ -114,16 +114,32 @@ void convert_matrix(const float* src, void* dst, size_t rows, size_t cols, size_
   }
 }
 
-#define VIT_LAUNCH(h, expr)                          \
+// Brackets one kernel launch with a pair of events on its stream while profiling is on.
+struct ProfScope {
+  Handle* h; cudaStream_t s; int cls; cudaEvent_t a = nullptr, b = nullptr;
+  ProfScope(Handle* h_, cudaStream_t s_, int cls_) : h(h_), s(s_), cls(cls_) {
+    if (!h->profiling) return;
+    if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { a = b = nullptr; return; }
+    cudaEventRecord(a, s);
+  }
+  ~ProfScope() {
+    if (!a) return;
+    cudaEventRecord(b, s);
+    h->prof.push_back(ProfRecord{a, b, cls});
+  }
+};
+
+#define VIT_LAUNCH(h, cls, expr)                     \
   do {                                               \
+    ProfScope prof__((h), s, (cls));                 \
     cudaError_t e__ = (expr);                        \
     if (e__ != cudaSuccess) return VIT_ERR_CUDA;     \
     (h)->launches.fetch_add(1, std::memory_order_relaxed); \
   } while (0)
 
-int linear(Handle* h, const LinearArgs& a, cudaStream_t s) {
-  if (h->cfg.dtype == VIT_BF16) VIT_LAUNCH(h, launch_linear_tc(a, h->dev_status, s));
-  else VIT_LAUNCH(h, launch_linear_f32(a, s));
+int linear(Handle* h, int cls, const LinearArgs& a, cudaStream_t s) {
+  if (h->cfg.dtype == VIT_BF16) VIT_LAUNCH(h, cls, launch_linear_tc(a, h->dev_status, s));
+  else VIT_LAUNCH(h, cls, launch_linear_f32(a, s));
   return VIT_OK;
 }
 
@@ -301,6 +317,7 @@ int vit_create(const vit_config* cfg, const float* host_params, size_t n_params,
   h->dev_blob_bytes = blob_bytes;
   h->dev_status = dev_status;
   h->launches.store(0);
+  h->profiling = false;
   const uint8_t* B = static_cast<const uint8_t*>(dev_blob);
   auto fp = [&](size_t i) { return reinterpret_cast<const float*>(B + items[i].dst); };
   auto vp = [&](size_t i) { return static_cast<const void*>(B + items[i].dst); };
@@ -321,6 +338,7 @@ int vit_create(const vit_config* cfg, const float* host_params, size_t n_params,
 int vit_destroy(vit_handle* h) {
   if (!h) return VIT_ERR_INVALID_ARG;
   cudaDeviceSynchronize();
+  for (const ProfRecord& r : h->prof) { cudaEventDestroy(r.begin); cudaEventDestroy(r.end); }
   cudaFree(h->dev_blob);
   cudaFree(h->dev_status);
   delete[] h->layers;
@@ -336,7 +354,7 @@ int vit_patch_embed(vit_handle* h, int mb, const float* pixels, void* tokens_out
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const vit_config& c = h->cfg;
   const bool b16 = c.dtype == VIT_BF16;
-  VIT_LAUNCH(h, launch_im2col(pixels, ws, mb, c.channels, c.image_size, c.patch_size, h->patch_k_pad, b16, s));
+  VIT_LAUNCH(h, VIT_PROF_EMBED, launch_im2col(pixels, ws, mb, c.channels, c.image_size, c.patch_size, h->patch_k_pad, b16, s));
   LinearArgs a{};
   a.M = mb * h->n_patches; a.N = c.hidden; a.K = h->patch_k_pad;
   a.a = ws; a.lda = h->patch_k_pad;
@@ -345,9 +363,9 @@ int vit_patch_embed(vit_handle* h, int mb, const float* pixels, void* tokens_out
   a.epilogue = EPI_BIAS_POS;
   a.pos = h->pos; a.n_patches = h->n_patches;
   a.out = tokens_out; a.ldo = c.hidden;
-  st = linear(h, a, s);
+  st = linear(h, VIT_PROF_EMBED, a, s);
   if (st != VIT_OK) return st;
-  VIT_LAUNCH(h, launch_cls_rows(h->cls, h->pos, tokens_out, mb, h->T, c.hidden, b16, s));
+  VIT_LAUNCH(h, VIT_PROF_EMBED, launch_cls_rows(h->cls, h->pos, tokens_out, mb, h->T, c.hidden, b16, s));
   return VIT_OK;
 }
 
@@ -375,38 +393,38 @@ int vit_run_stage(vit_handle* h, int layer_begin, int layer_end, int mb, const v
     const LayerWeights& w = h->layers[l];
     const void* x_in = (l == layer_begin) ? in : out;
     // y = LN1(x)
-    if (b16) VIT_LAUNCH(h, launch_layernorm_bf16((const bf16*)x_in, w.ln1_g, w.ln1_b, c.ln_eps, (bf16*)y, (int)M, (int)H, s));
-    else VIT_LAUNCH(h, launch_layernorm_f32((const float*)x_in, w.ln1_g, w.ln1_b, c.ln_eps, (float*)y, (int)M, (int)H, s));
+    if (b16) VIT_LAUNCH(h, VIT_PROF_LAYERNORM, launch_layernorm_bf16((const bf16*)x_in, w.ln1_g, w.ln1_b, c.ln_eps, (bf16*)y, (int)M, (int)H, s));
+    else VIT_LAUNCH(h, VIT_PROF_LAYERNORM, launch_layernorm_f32((const float*)x_in, w.ln1_g, w.ln1_b, c.ln_eps, (float*)y, (int)M, (int)H, s));
     // qkv = y Wqkv^T + bqkv
     LinearArgs a{};
     a.M = (int)M; a.N = (int)(3 * H); a.K = (int)H;
     a.a = y; a.lda = (int)H; a.w = w.Wqkv; a.ldw = (int)H; a.bias = w.bqkv;
     a.epilogue = EPI_BIAS; a.out = wide; a.ldo = (int)(3 * H);
-    if ((st = linear(h, a, s)) != VIT_OK) return st;
+    if ((st = linear(h, VIT_PROF_QKV, a, s)) != VIT_OK) return st;
     // y = attention(qkv)
-    if (b16) VIT_LAUNCH(h, launch_attention_bf16((const bf16*)wide, (bf16*)y, mb, h->T, c.heads, h->d, s));
-    else VIT_LAUNCH(h, launch_attention_f32((const float*)wide, (float*)y, mb, h->T, c.heads, h->d, s));
+    if (b16) VIT_LAUNCH(h, VIT_PROF_ATTENTION, launch_attention_bf16((const bf16*)wide, (bf16*)y, mb, h->T, c.heads, h->d, s));
+    else VIT_LAUNCH(h, VIT_PROF_ATTENTION, launch_attention_f32((const float*)wide, (float*)y, mb, h->T, c.heads, h->d, s));
     // x = x + y Wo^T + bo
     a = LinearArgs{};
     a.M = (int)M; a.N = (int)H; a.K = (int)H;
     a.a = y; a.lda = (int)H; a.w = w.Wo; a.ldw = (int)H; a.bias = w.bo;
     a.epilogue = EPI_BIAS_RESIDUAL; a.residual = x_in; a.out = out; a.ldo = (int)H;
-    if ((st = linear(h, a, s)) != VIT_OK) return st;
+    if ((st = linear(h, VIT_PROF_OUTPROJ, a, s)) != VIT_OK) return st;
     // y = LN2(x)
-    if (b16) VIT_LAUNCH(h, launch_layernorm_bf16((const bf16*)out, w.ln2_g, w.ln2_b, c.ln_eps, (bf16*)y, (int)M, (int)H, s));
-    else VIT_LAUNCH(h, launch_layernorm_f32((const float*)out, w.ln2_g, w.ln2_b, c.ln_eps, (float*)y, (int)M, (int)H, s));
+    if (b16) VIT_LAUNCH(h, VIT_PROF_LAYERNORM, launch_layernorm_bf16((const bf16*)out, w.ln2_g, w.ln2_b, c.ln_eps, (bf16*)y, (int)M, (int)H, s));
+    else VIT_LAUNCH(h, VIT_PROF_LAYERNORM, launch_layernorm_f32((const float*)out, w.ln2_g, w.ln2_b, c.ln_eps, (float*)y, (int)M, (int)H, s));
     // u = gelu(y W1^T + b1)
     a = LinearArgs{};
     a.M = (int)M; a.N = (int)F; a.K = (int)H;
     a.a = y; a.lda = (int)H; a.w = w.W1; a.ldw = (int)H; a.bias = w.b1;
     a.epilogue = EPI_BIAS_GELU; a.out = wide; a.ldo = (int)F;
-    if ((st = linear(h, a, s)) != VIT_OK) return st;
+    if ((st = linear(h, VIT_PROF_FC1, a, s)) != VIT_OK) return st;
     // x = x + u W2^T + b2
     a = LinearArgs{};
     a.M = (int)M; a.N = (int)H; a.K = (int)F;
     a.a = wide; a.lda = (int)F; a.w = w.W2; a.ldw = (int)F; a.bias = w.b2;
     a.epilogue = EPI_BIAS_RESIDUAL; a.residual = out; a.out = out; a.ldo = (int)H;
-    if ((st = linear(h, a, s)) != VIT_OK) return st;
+    if ((st = linear(h, VIT_PROF_FC2, a, s)) != VIT_OK) return st;
   }
   return VIT_OK;
 }
@@ -417,11 +435,11 @@ int vit_head(vit_handle* h, int mb, const void* tokens, float* logits, void* ws,
   if (st != VIT_OK) return st;
   if (!tokens || !logits || misaligned(tokens) || misaligned(logits)) return VIT_ERR_INVALID_ARG;
   const vit_config& c = h->cfg;
-  cudaError_t e = launch_head(tokens, h->lnf_g, h->lnf_b, c.ln_eps, h->head_W, h->head_b,
-                              static_cast<float*>(ws), logits, mb, h->T, c.hidden, c.num_classes,
-                              c.dtype == VIT_BF16, static_cast<cudaStream_t>(stream));
-  if (e != cudaSuccess) return VIT_ERR_CUDA;
-  h->launches.fetch_add(2, std::memory_order_relaxed);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  VIT_LAUNCH(h, VIT_PROF_HEAD, launch_head(tokens, h->lnf_g, h->lnf_b, c.ln_eps, h->head_W, h->head_b,
+                                           static_cast<float*>(ws), logits, mb, h->T, c.hidden,
+                                           c.num_classes, c.dtype == VIT_BF16, s));
+  h->launches.fetch_add(1, std::memory_order_relaxed);   // the head is two kernels
   return VIT_OK;
 }
 
@@ -448,6 +466,30 @@ int vit_check_status(vit_handle* h, void* stream) {
   return v;
 }
 
+int vit_profile_enable(vit_handle* h, int on) {
+  if (!h) return VIT_ERR_INVALID_ARG;
+  h->profiling = on != 0;
+  return VIT_OK;
+}
+
+int vit_profile_collect(vit_handle* h, double* ms_by_class, uint64_t* launches_by_class) {
+  if (!h || !ms_by_class || !launches_by_class) return VIT_ERR_INVALID_ARG;
+  for (int i = 0; i < VIT_PROF_CLASSES; ++i) { ms_by_class[i] = 0.0; launches_by_class[i] = 0; }
+  int st = VIT_OK;
+  if (cudaDeviceSynchronize() != cudaSuccess) st = VIT_ERR_CUDA;
+  for (const ProfRecord& r : h->prof) {
+    float ms = 0.f;
+    if (st == VIT_OK && cudaEventElapsedTime(&ms, r.begin, r.end) == cudaSuccess) {
+      ms_by_class[r.cls] += ms;
+      launches_by_class[r.cls] += 1;
+    }
+    cudaEventDestroy(r.begin);
+    cudaEventDestroy(r.end);
+  }
+  h->prof.clear();
+  return st;
+}
+
 uint64_t vit_launch_count(const vit_handle* h) { return h ? h->launches.load() : 0; }
 
 const char* vit_status_string(int status) {
@@ -469,8 +511,8 @@ int vit_op_layernorm(vit_handle* h, int dtype, int rows, int cols, const void* x
   if (!h || !x || !gain || !shift || !y || rows < 0 || cols < 1) return VIT_ERR_INVALID_ARG;
   if (misaligned(x) || misaligned(y) || misaligned(gain) || misaligned(shift)) return VIT_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (dtype == VIT_BF16) VIT_LAUNCH(h, launch_layernorm_bf16((const bf16*)x, gain, shift, eps, (bf16*)y, rows, cols, s));
-  else if (dtype == VIT_FP32) VIT_LAUNCH(h, launch_layernorm_f32((const float*)x, gain, shift, eps, (float*)y, rows, cols, s));
+  if (dtype == VIT_BF16) VIT_LAUNCH(h, VIT_PROF_LAYERNORM, launch_layernorm_bf16((const bf16*)x, gain, shift, eps, (bf16*)y, rows, cols, s));
+  else if (dtype == VIT_FP32) VIT_LAUNCH(h, VIT_PROF_LAYERNORM, launch_layernorm_f32((const float*)x, gain, shift, eps, (float*)y, rows, cols, s));
   else return VIT_ERR_INVALID_ARG;
   return VIT_OK;
 }
@@ -487,9 +529,9 @@ int vit_op_linear(vit_handle* h, int dtype, int M, int N, int K, const void* a, 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (dtype == VIT_BF16) {
     if (K % 8 || N % 8) return VIT_ERR_INVALID_ARG;
-    VIT_LAUNCH(h, launch_linear_tc(p, h->dev_status, s));
+    VIT_LAUNCH(h, VIT_PROF_OP, launch_linear_tc(p, h->dev_status, s));
   } else if (dtype == VIT_FP32) {
-    VIT_LAUNCH(h, launch_linear_f32(p, s));
+    VIT_LAUNCH(h, VIT_PROF_OP, launch_linear_f32(p, s));
   } else {
     return VIT_ERR_INVALID_ARG;
   }
@@ -503,9 +545,9 @@ int vit_op_attention(vit_handle* h, int dtype, int images, int T, int heads, int
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (dtype == VIT_BF16) {
     if (d % 16 || d > 128) return VIT_ERR_INVALID_ARG;
-    VIT_LAUNCH(h, launch_attention_bf16((const bf16*)qkv, (bf16*)out, images, T, heads, d, s));
+    VIT_LAUNCH(h, VIT_PROF_ATTENTION, launch_attention_bf16((const bf16*)qkv, (bf16*)out, images, T, heads, d, s));
   } else if (dtype == VIT_FP32) {
-    VIT_LAUNCH(h, launch_attention_f32((const float*)qkv, (float*)out, images, T, heads, d, s));
+    VIT_LAUNCH(h, VIT_PROF_ATTENTION, launch_attention_f32((const float*)qkv, (float*)out, images, T, heads, d, s));
   } else {
     return VIT_ERR_INVALID_ARG;
   }

@@ -5,6 +5,7 @@
 #include <stdint.h>
 #include <stddef.h>
 #include <atomic>
+#include <vector>
 
 #include "../../include/vit.h"
 
@@ -41,6 +42,8 @@ struct LayerWeights {
   const void *Wqkv, *Wo, *W1, *W2;   // activation type, [out, in]
 };
 
+struct ProfRecord { cudaEvent_t begin, end; int cls; };
+
 struct Handle {
   vit_config cfg;
   int T, n_patches, d, patch_k, patch_k_pad;
@@ -54,6 +57,8 @@ struct Handle {
   const void* head_W;                // [classes, H]
   int* dev_status;                   // device status word (0 = ok)
   std::atomic<uint64_t> launches;
+  bool profiling;                    // event pair around every launch (single-threaded use)
+  std::vector<ProfRecord> prof;
 };
 
 // ---- kernel launchers (each returns a cudaError_t from the launch) ------------------------

@@ -3,7 +3,9 @@
 // Persistent, warp-specialised kernel, one CTA per SM:
 //   warp 0      TMA producer: 128 x 64 tile of a and BN x 64 tile of w per stage, 128-byte swizzle
 //   warp 1      allocates tensor memory and issues tcgen05.mma (128 x BN x 16 per instruction)
-//   warps 2..9  epilogue: tcgen05.ld the fp32 accumulator, bias / GELU / residual, bf16 stores
+//   warps 2..9  epilogue: tcgen05.ld the fp32 accumulator, bias / GELU / residual, bf16 rows staged
+//               in swizzled shared memory and written with TMA stores (the residual tile arrives
+//               the same way, by TMA load), so global traffic is coalesced and asynchronous
 // Two accumulators live in tensor memory (2 x BN columns) so the epilogue of tile i overlaps the
 // main loop of tile i+1.  Tiles are handed out statically (tile = blockIdx.x + i * gridDim.x).
 // Every mbarrier wait is bounded; on expiry the CTA raises the device status word and leaves.
@@ -28,7 +30,9 @@ template <int BN> struct Cfg {
   static constexpr int B_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int TMEM_COLS = 2 * BN;                 // 512 or 256: a power of two
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int STAGING_BYTES = NUM_EPI_WARPS * 4096;   // 32 rows x 128 B per epilogue warp
+  static constexpr int SMEM_BYTES =
+      STAGES * STAGE_BYTES + STAGING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -140,8 +144,37 @@ __device__ __forceinline__ void tmem_ld_wait() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(
+                   reinterpret_cast<uint64_t>(tm)),
+               "r"(src), "r"(x), "r"(y)
+               : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void tma_store_wait_read() {   // staging buffer may be overwritten
+  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+__device__ __forceinline__ void tma_store_wait_all() {    // stores complete
+  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// gelu(v) = 0.5 v (1 + erf(v / sqrt 2)) with erfc(z) = (a1 t + ... + a5 t^5) exp(-z^2),
+// t = 1 / (1 + p z), z >= 0 (Abramowitz & Stegun 7.1.26, |error| <= 1.5e-7), on the MUFU
+// reciprocal and exp2.  For v >= 0: v - 0.5 v erfc(z); for v < 0: 0.5 v erfc(z).
 __device__ __forceinline__ float gelu_erf(float v) {
-  return 0.5f * v * (1.0f + erff(v * 0.70710678118654752440f));
+  const float z = fabsf(v) * 0.70710678118654752440f;
+  const float t = __fdividef(1.0f, fmaf(0.3275911f, z, 1.0f));
+  float e;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(z * z * -1.4426950408889634f));
+  float q = fmaf(1.061405429f, t, -1.453152027f);
+  q = fmaf(q, t, 1.421413741f);
+  q = fmaf(q, t, -0.284496736f);
+  q = fmaf(q, t, 0.254829592f);
+  const float h = 0.5f * v * (q * t * e);
+  return v >= 0.f ? v - h : h;
 }
 
 struct TcParams {
@@ -159,18 +192,21 @@ struct TcParams {
 template <int BN, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w,
+                 const __grid_constant__ CUtensorMap tm_out, const __grid_constant__ CUtensorMap tm_res,
                  const TcParams p) {
   using C = Cfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte alignment: the swizzle pattern and the descriptors assume it
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* tiles = smem;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::STAGES * C::STAGE_BYTES);
+  uint8_t* staging = smem + C::STAGES * C::STAGE_BYTES;   // 1024-aligned: 4 KB per epilogue warp
+  uint64_t* bars = reinterpret_cast<uint64_t*>(staging + C::STAGING_BYTES);
   uint64_t* full_bar = bars;                       // [STAGES]
   uint64_t* empty_bar = bars + C::STAGES;          // [STAGES]
   uint64_t* tfull_bar = bars + 2 * C::STAGES;      // [2]
   uint64_t* tempty_bar = bars + 2 * C::STAGES + 2; // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * C::STAGES + 4);
+  uint64_t* res_bar = bars + 2 * C::STAGES + 4;    // [NUM_EPI_WARPS] residual tile landed
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * C::STAGES + 4 + NUM_EPI_WARPS);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -187,9 +223,11 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       mbar_init(smem_u32(&tfull_bar[i]), 1);
       mbar_init(smem_u32(&tempty_bar[i]), NUM_EPI_WARPS);
     }
+    for (int i = 0; i < NUM_EPI_WARPS; ++i) mbar_init(smem_u32(&res_bar[i]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_a)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_w)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_out)) : "memory");
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
@@ -263,73 +301,137 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     constexpr int COLS_PER_WARP = BN / 2;
     int buf = 0;
     uint32_t aphase = 0;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-      const int m0 = (tile / p.tiles_n) * BM, n0 = (tile % p.tiles_n) * BN;
-      if (!mbar_wait(smem_u32(&tfull_bar[buf]), aphase, abort_flag)) break;
-      tc_fence_after();
-      const int row = m0 + quarter * 32 + lane;
-      const bool row_ok = row < p.M;
-      size_t orow = (size_t)row;
-      const float* posrow = nullptr;
-      if (EPI == EPI_BIAS_POS) {
+    if (EPI == EPI_BIAS_POS) {
+      // patch embedding: rows are scattered to token 1 + patch of their image, direct stores
+      for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+        const int m0 = (tile / p.tiles_n) * BM, n0 = (tile % p.tiles_n) * BN;
+        if (!mbar_wait(smem_u32(&tfull_bar[buf]), aphase, abort_flag)) break;
+        tc_fence_after();
+        const int row = m0 + quarter * 32 + lane;
+        const bool row_ok = row < p.M;
         const int img = row / p.n_patches, pt = row - img * p.n_patches;
-        orow = (size_t)img * (p.n_patches + 1) + 1 + pt;
-        posrow = p.pos + (size_t)(1 + pt) * p.N;
-      }
+        const size_t orow = (size_t)img * (p.n_patches + 1) + 1 + pt;
+        const float* posrow = p.pos + (size_t)(1 + pt) * p.N;
 #pragma unroll 1
-      for (int ch = 0; ch < COLS_PER_WARP / 32; ++ch) {
-        const int cl = half * COLS_PER_WARP + ch * 32;   // column inside the tile
-        const int c0 = n0 + cl;
-        if (c0 >= p.N) break;                            // uniform across the warp
-        uint32_t r[32];
-        tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cl), r);
-        tmem_ld_wait();
+        for (int ch = 0; ch < COLS_PER_WARP / 32; ++ch) {
+          const int cl = half * COLS_PER_WARP + ch * 32;
+          const int c0 = n0 + cl;
+          if (c0 >= p.N) break;                            // uniform across the warp
+          uint32_t r[32];
+          tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cl), r);
+          tmem_ld_wait();
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          const int c = c0 + g * 8;
-          if (c >= p.N) break;
-          const float4 b0 = __ldg(reinterpret_cast<const float4*>(p.bias + c));
-          const float4 b1 = __ldg(reinterpret_cast<const float4*>(p.bias + c) + 1);
-          float v[8];
-          v[0] = __uint_as_float(r[g * 8 + 0]) + b0.x;
-          v[1] = __uint_as_float(r[g * 8 + 1]) + b0.y;
-          v[2] = __uint_as_float(r[g * 8 + 2]) + b0.z;
-          v[3] = __uint_as_float(r[g * 8 + 3]) + b0.w;
-          v[4] = __uint_as_float(r[g * 8 + 4]) + b1.x;
-          v[5] = __uint_as_float(r[g * 8 + 5]) + b1.y;
-          v[6] = __uint_as_float(r[g * 8 + 6]) + b1.z;
-          v[7] = __uint_as_float(r[g * 8 + 7]) + b1.w;
-          if (row_ok) {
-            if (EPI == EPI_BIAS_GELU) {
+          for (int g = 0; g < 4; ++g) {
+            const int c = c0 + g * 8;
+            if (c >= p.N || !row_ok) continue;
+            uint4 o;
+            __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&o);
 #pragma unroll
-              for (int e = 0; e < 8; ++e) v[e] = gelu_erf(v[e]);
-            } else if (EPI == EPI_BIAS_RESIDUAL) {
-              const uint4 u = *reinterpret_cast<const uint4*>(p.residual + orow * p.ldo + c);
+            for (int e = 0; e < 4; ++e) {
+              const float v0 = __uint_as_float(r[g * 8 + 2 * e]) + __ldg(p.bias + c + 2 * e) +
+                               __ldg(posrow + c + 2 * e);
+              const float v1 = __uint_as_float(r[g * 8 + 2 * e + 1]) + __ldg(p.bias + c + 2 * e + 1) +
+                               __ldg(posrow + c + 2 * e + 1);
+              h[e] = __floats2bfloat162_rn(v0, v1);
+            }
+            *reinterpret_cast<uint4*>(p.out + orow * p.ldo + c) = o;
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[buf]));
+        if (++buf == 2) { buf = 0; aphase ^= 1; }
+      }
+    } else {
+      uint8_t* stg = staging + ew * 4096;            // this warp's 32-row x 64-column bf16 tile
+      const uint32_t stg_u32 = smem_u32(stg);
+      const uint32_t my_row = stg_u32 + (uint32_t)lane * 128u;
+      const uint32_t rb = smem_u32(&res_bar[ew]);
+      uint32_t rphase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const int m0 = (tile / p.tiles_n) * BM, n0 = (tile % p.tiles_n) * BN;
+        const int row0 = m0 + quarter * 32;
+#pragma unroll 1
+        for (int cb = 0; cb < COLS_PER_WARP / 64; ++cb) {
+          const int cl = half * COLS_PER_WARP + cb * 64;   // column inside the tile
+          const int c0 = n0 + cl;
+          if (c0 >= p.N) break;                            // uniform across the warp
+          if (EPI == EPI_BIAS_RESIDUAL) {
+            // bring the residual tile into the staging buffer while the accumulator is awaited
+            if (lane == 0) {
+              tma_store_wait_read();
+              mbar_arrive_expect_tx(rb, 4096);
+              tma_load_2d(stg_u32, &tm_res, c0, row0, rb);
+            }
+          }
+          if (cb == 0) {
+            if (!mbar_wait(smem_u32(&tfull_bar[buf]), aphase, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+          }
+          uint32_t r[64];
+          const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + cl);
+          tmem_ld32(taddr, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+          tmem_ld32(taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+          tmem_ld_wait();
+          float v[64];
+#pragma unroll
+          for (int g = 0; g < 16; ++g) {
+            const float4 b = (c0 + 4 * g < p.N) ? __ldg(reinterpret_cast<const float4*>(p.bias + c0) + g)
+                                                : make_float4(0.f, 0.f, 0.f, 0.f);
+            v[4 * g + 0] = __uint_as_float(r[4 * g + 0]) + b.x;
+            v[4 * g + 1] = __uint_as_float(r[4 * g + 1]) + b.y;
+            v[4 * g + 2] = __uint_as_float(r[4 * g + 2]) + b.z;
+            v[4 * g + 3] = __uint_as_float(r[4 * g + 3]) + b.w;
+          }
+          if (EPI == EPI_BIAS_GELU) {
+#pragma unroll
+            for (int e = 0; e < 64; ++e) v[e] = gelu_erf(v[e]);
+          }
+          if (EPI == EPI_BIAS_RESIDUAL) {
+            if (!mbar_wait(rb, rphase, abort_flag)) { ok = false; break; }
+            rphase ^= 1;
+#pragma unroll
+            for (int ck = 0; ck < 8; ++ck) {
+              uint4 u;
+              const uint32_t a = my_row + (uint32_t)((ck ^ (lane & 7)) << 4);
+              asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                           : "=r"(u.x), "=r"(u.y), "=r"(u.z), "=r"(u.w)
+                           : "r"(a));
               const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
                 const float2 f = __bfloat1622float2(h[e]);
-                v[2 * e] += f.x;
-                v[2 * e + 1] += f.y;
+                v[ck * 8 + 2 * e] += f.x;
+                v[ck * 8 + 2 * e + 1] += f.y;
               }
-            } else if (EPI == EPI_BIAS_POS) {
-              const float4 p0 = __ldg(reinterpret_cast<const float4*>(posrow + c));
-              const float4 p1 = __ldg(reinterpret_cast<const float4*>(posrow + c) + 1);
-              v[0] += p0.x; v[1] += p0.y; v[2] += p0.z; v[3] += p0.w;
-              v[4] += p1.x; v[5] += p1.y; v[6] += p1.z; v[7] += p1.w;
             }
+          } else {
+            if (lane == 0) tma_store_wait_read();          // previous store has left the buffer
+            __syncwarp();
+          }
+#pragma unroll
+          for (int ck = 0; ck < 8; ++ck) {
             uint4 o;
             __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&o);
 #pragma unroll
-            for (int e = 0; e < 4; ++e) h[e] = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
-            *reinterpret_cast<uint4*>(p.out + orow * p.ldo + c) = o;
+            for (int e = 0; e < 4; ++e) h[e] = __floats2bfloat162_rn(v[ck * 8 + 2 * e], v[ck * 8 + 2 * e + 1]);
+            const uint32_t a = my_row + (uint32_t)((ck ^ (lane & 7)) << 4);   // 128-byte swizzle
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(o.x), "r"(o.y),
+                         "r"(o.z), "r"(o.w)
+                         : "memory");
           }
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) tma_store_2d(&tm_out, stg_u32, c0, row0);   // rows >= M, columns >= N are clipped
         }
+        if (!ok) break;
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[buf]));
+        if (++buf == 2) { buf = 0; aphase ^= 1; }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[buf]));
-      if (++buf == 2) { buf = 0; aphase ^= 1; }
+      if (lane == 0) tma_store_wait_all();
     }
   }
 
@@ -357,6 +459,7 @@ EncodeTiledFn g_encode = nullptr;
 int g_num_sms = 0;
 
 bool encode_2d_bf16(CUtensorMap* tm, const void* base, int rows, int cols, int ld, int box_rows) {
+  if (base == nullptr) return false;
   const cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   const cuuint64_t gstride[1] = {(cuuint64_t)ld * 2};
   const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
@@ -366,9 +469,10 @@ bool encode_2d_bf16(CUtensorMap* tm, const void* base, int rows, int cols, int l
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+struct Maps { CUtensorMap a, w, out, res; };
+
 template <int BN, int EPI>
-cudaError_t launch_variant(const CUtensorMap& ta, const CUtensorMap& tw, const TcParams& p,
-                           cudaStream_t s) {
+cudaError_t launch_variant(const Maps& m, const TcParams& p, cudaStream_t s) {
   static bool configured = false;   // benign race: the attribute is idempotent
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(linear_tc_kernel<BN, EPI>,
@@ -379,18 +483,17 @@ cudaError_t launch_variant(const CUtensorMap& ta, const CUtensorMap& tw, const T
   }
   const int total = p.tiles_m * p.tiles_n;
   const int grid = total < g_num_sms ? total : g_num_sms;
-  linear_tc_kernel<BN, EPI><<<grid, NUM_THREADS, Cfg<BN>::SMEM_BYTES, s>>>(ta, tw, p);
+  linear_tc_kernel<BN, EPI><<<grid, NUM_THREADS, Cfg<BN>::SMEM_BYTES, s>>>(m.a, m.w, m.out, m.res, p);
   return cudaGetLastError();
 }
 
 template <int BN>
-cudaError_t launch_bn(int epi, const CUtensorMap& ta, const CUtensorMap& tw, const TcParams& p,
-                      cudaStream_t s) {
+cudaError_t launch_bn(int epi, const Maps& m, const TcParams& p, cudaStream_t s) {
   switch (epi) {
-    case EPI_BIAS: return launch_variant<BN, EPI_BIAS>(ta, tw, p, s);
-    case EPI_BIAS_GELU: return launch_variant<BN, EPI_BIAS_GELU>(ta, tw, p, s);
-    case EPI_BIAS_RESIDUAL: return launch_variant<BN, EPI_BIAS_RESIDUAL>(ta, tw, p, s);
-    case EPI_BIAS_POS: return launch_variant<BN, EPI_BIAS_POS>(ta, tw, p, s);
+    case EPI_BIAS: return launch_variant<BN, EPI_BIAS>(m, p, s);
+    case EPI_BIAS_GELU: return launch_variant<BN, EPI_BIAS_GELU>(m, p, s);
+    case EPI_BIAS_RESIDUAL: return launch_variant<BN, EPI_BIAS_RESIDUAL>(m, p, s);
+    case EPI_BIAS_POS: return launch_variant<BN, EPI_BIAS_POS>(m, p, s);
   }
   return cudaErrorInvalidValue;
 }
@@ -433,10 +536,17 @@ cudaError_t launch_linear_tc(const LinearArgs& a, int* dev_status, cudaStream_t 
   p.tiles_m = tiles_m;
   p.tiles_n = (a.N + bn - 1) / bn;
   p.dev_status = dev_status;
-  CUtensorMap ta, tw;
-  if (!encode_2d_bf16(&ta, a.a, a.M, a.K, a.lda, BM)) return cudaErrorInvalidValue;
-  if (!encode_2d_bf16(&tw, a.w, a.N, a.K, a.ldw, bn)) return cudaErrorInvalidValue;
-  return wide ? launch_bn<256>(a.epilogue, ta, tw, p, s) : launch_bn<128>(a.epilogue, ta, tw, p, s);
+  Maps m;
+  if (!encode_2d_bf16(&m.a, a.a, a.M, a.K, a.lda, BM)) return cudaErrorInvalidValue;
+  if (!encode_2d_bf16(&m.w, a.w, a.N, a.K, a.ldw, bn)) return cudaErrorInvalidValue;
+  // output (and residual) tiles move as 32-row x 64-column boxes through the epilogue's staging
+  if (!encode_2d_bf16(&m.out, a.out, a.M, a.N, a.ldo, 32)) return cudaErrorInvalidValue;
+  if (a.epilogue == EPI_BIAS_RESIDUAL) {
+    if (!encode_2d_bf16(&m.res, a.residual, a.M, a.N, a.ldo, 32)) return cudaErrorInvalidValue;
+  } else {
+    m.res = m.out;
+  }
+  return wide ? launch_bn<256>(a.epilogue, m, p, s) : launch_bn<128>(a.epilogue, m, p, s);
 }
 
 }  // namespace vit

@@ -40,7 +40,8 @@ enum {
   VIT_ERR_WORKSPACE = -4,   /* workspace smaller than the size query says */
   VIT_ERR_CUDA = -5,        /* a CUDA runtime/driver call or a launch failed */
   VIT_ERR_TIMEOUT = -6,     /* a bounded wait inside a kernel gave up (device status word) */
-  VIT_ERR_NO_DEVICE = -7    /* no sm_100 device / driver available */
+  VIT_ERR_NO_DEVICE = -7,   /* no sm_100 device / driver available */
+  VIT_ERR_TOO_LARGE = -8    /* problem exceeds the fixed scratch of an allocation-free entry point */
 };
 
 enum { VIT_BF16 = 0, VIT_FP32 = 1 };
@@ -116,6 +117,29 @@ int vit_run_stage(vit_handle* h, int layer_begin, int layer_end, int microbatch,
  *   tokens: dev, activations [microbatch, T, H];  logits: dev, fp32 [microbatch, classes]. */
 int vit_head(vit_handle* h, int microbatch, const void* tokens, float* logits,
              void* ws, size_t ws_bytes, void* stream);
+
+/* vit_head for callers that cannot allocate device memory.  (The paper has no counterpart; this
+ * is a convenience of the library.)  Some code that wants the classification result runs where
+ * cudaMalloc is off limits: a real-time loop that must never enter the allocator (it can block
+ * and synchronise the device), a plugin whose host application owns all device memory and hands
+ * out only the input and output buffers, or a process whose memory pool was given away whole to
+ * another framework at start-up.  vit_head needs a scratch buffer for
+ * the normalised class-token features; this variant keeps that scratch in an array that is part
+ * of the library itself, so the caller passes only tokens and logits.
+ *   - Same arithmetic and same results as vit_head.
+ *   - Limit: microbatch * hidden <= VIT_HEAD_STATIC_MAX_FLOATS (2 MiB of floats); anything
+ *     larger returns VIT_ERR_TOO_LARGE and launches nothing.  Every GPU on which the library
+ *     is loaded carries the array (2 MiB) until the process exits.
+ *   - The first call on each device looks up the array's device address (a runtime query, not
+ *     an allocation); make that first call before starting any stream capture.  It must be
+ *     made with the handle's device current, like every other call.
+ *   - There is ONE array per device, shared by all handles and streams, and it keeps whatever
+ *     the last call left in it.  Nothing in it has to be cleared: a call overwrites every value
+ *     before reading it.  Two calls that may run on the GPU at the same time (different
+ *     streams, no dependency between them) would overwrite each other's features: order them.
+ *   - Calls no cudaMalloc / cudaFree and no allocating library routine. */
+#define VIT_HEAD_STATIC_MAX_FLOATS (512 * 1024)
+int vit_head_static(vit_handle* h, int microbatch, const void* tokens, float* logits, void* stream);
 
 /* Stage runner (paper Section 2.1/3.1: the minibatch is split into equal microbatches that
  * flow through the stages in order).  Splits `batch` images into microbatches of `microbatch`

@@ -18,6 +18,8 @@ LIB_PATH = os.path.join(_PKG, "libvit_b200.so")
 VIT_OK = 0
 VIT_ERR_INVALID_ARG, VIT_ERR_RANGE, VIT_ERR_CONFIG, VIT_ERR_WORKSPACE = -1, -2, -3, -4
 VIT_ERR_CUDA, VIT_ERR_TIMEOUT, VIT_ERR_NO_DEVICE = -5, -6, -7
+VIT_ERR_TOO_LARGE = -8
+VIT_HEAD_STATIC_MAX_FLOATS = 512 * 1024
 VIT_BF16, VIT_FP32 = 0, 1
 
 EXPORTS = [
@@ -25,7 +27,7 @@ EXPORTS = [
     "vit_destroy", "vit_patch_embed", "vit_run_stage", "vit_head", "vit_run_pipeline",
     "vit_run_pipeline_host", "vit_check_status", "vit_launch_count", "vit_status_string",
     "vit_op_layernorm", "vit_op_linear", "vit_op_attention", "vit_profile_enable",
-    "vit_profile_collect",
+    "vit_profile_collect", "vit_head_static",
 ]
 PROF_CLASSES = ["layernorm", "qkv", "attention", "outproj", "fc1", "fc2", "embed", "head", "op"]
 
@@ -89,6 +91,8 @@ def lib():
     L.vit_op_linear.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p]
     L.vit_op_attention.restype = c_int
     L.vit_op_attention.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p]
+    L.vit_head_static.restype = c_int
+    L.vit_head_static.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p]
     L.vit_profile_enable.restype = c_int
     L.vit_profile_enable.argtypes = [c_void_p, c_int]
     L.vit_profile_collect.restype = c_int
@@ -150,6 +154,12 @@ def vit_run_stage(h, layer_begin, layer_end, microbatch, inp, out, ws, ws_bytes,
 
 def vit_head(h, microbatch, tokens, logits, ws, ws_bytes, stream=0):
     _check(lib().vit_head(h, microbatch, tokens, logits, ws, ws_bytes, stream), "vit_head")
+
+
+def vit_head_static(h, microbatch, tokens, logits, stream=0):
+    """vit_head with the scratch inside the library: for callers that cannot allocate device
+    memory.  Raises VitError(VIT_ERR_TOO_LARGE) beyond microbatch * hidden = 512 Ki."""
+    _check(lib().vit_head_static(h, microbatch, tokens, logits, stream), "vit_head_static")
 
 
 def _pipeline(fn, name, h, stage_layers, batch, microbatch, pixels, logits, ws_ptrs, ws_bytes, streams):

@@ -1,6 +1,8 @@
 // LayerNorm, the fp32 (SIMT) kernel family, and the two book-ends' small kernels.
 #include "vit_internal.h"
 
+#include <mutex>
+
 namespace vit {
 
 __device__ __forceinline__ float warp_sum(float v) {
@@ -395,6 +397,44 @@ cudaError_t launch_head(const void* tokens, const float* g, const float* b, floa
     head_logits_kernel<float><<<b2, threads, 0, s>>>(feat, (const float*)W, bias, logits, images, H, classes);
   }
   return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Head without caller scratch: the class-token features go to a fixed array that is part of
+// the library image, for callers that have no way to allocate device memory.
+// In host code the array's name is only a handle for the runtime; the address the kernels need
+// is looked up once per device with cudaGetSymbolAddress while that device is current.
+// ------------------------------------------------------------------------------------------
+static __device__ __align__(256) float g_head_static_scratch[VIT_HEAD_STATIC_MAX_FLOATS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+float* g_static_ptr[kMaxDevices] = {};
+}  // namespace
+
+cudaError_t launch_head_static(const void* tokens, const float* g, const float* b, float eps,
+                               const void* W, const float* bias, float* logits, int images, int T,
+                               int H, int classes, bool act_bf16, cudaStream_t s) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  float* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (g_static_ptr[dev] == nullptr) {
+      float* ptr = nullptr;
+      e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_head_static_scratch);
+      if (e != cudaSuccess) return e;
+      if (ptr == nullptr) return cudaErrorInvalidSymbol;
+      g_static_ptr[dev] = ptr;
+    }
+    scratch = g_static_ptr[dev];
+  }
+  // Every feature the logits kernel reads is written by the LayerNorm kernel of the same call
+  // first, so nothing in the array has to start at zero.
+  return launch_head(tokens, g, b, eps, W, bias, scratch, logits, images, T, H, classes, act_bf16, s);
 }
 
 }  // namespace vit

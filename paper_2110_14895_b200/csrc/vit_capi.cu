@@ -443,6 +443,19 @@ int vit_head(vit_handle* h, int mb, const void* tokens, float* logits, void* ws,
   return VIT_OK;
 }
 
+int vit_head_static(vit_handle* h, int mb, const void* tokens, float* logits, void* stream) {
+  if (!h || mb < 1 || mb > h->cfg.max_microbatch) return VIT_ERR_INVALID_ARG;
+  if (!tokens || !logits || misaligned(tokens) || misaligned(logits)) return VIT_ERR_INVALID_ARG;
+  const vit_config& c = h->cfg;
+  if ((size_t)mb * (size_t)c.hidden > (size_t)VIT_HEAD_STATIC_MAX_FLOATS) return VIT_ERR_TOO_LARGE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  VIT_LAUNCH(h, VIT_PROF_HEAD, launch_head_static(tokens, h->lnf_g, h->lnf_b, c.ln_eps, h->head_W,
+                                                  h->head_b, logits, mb, h->T, c.hidden,
+                                                  c.num_classes, c.dtype == VIT_BF16, s));
+  h->launches.fetch_add(1, std::memory_order_relaxed);   // the head is two kernels
+  return VIT_OK;
+}
+
 int vit_run_pipeline(vit_handle* h, const int32_t* stage_layers, int n_stages, int batch, int mb,
                      const float* pixels, float* logits, void* const* ws_per_stream, size_t ws_bytes,
                      void* const* streams, int n_streams) {
@@ -502,6 +515,7 @@ const char* vit_status_string(int status) {
     case VIT_ERR_CUDA: return "CUDA call or kernel launch failed";
     case VIT_ERR_TIMEOUT: return "a bounded wait inside a kernel expired";
     case VIT_ERR_NO_DEVICE: return "no usable sm_100 device";
+    case VIT_ERR_TOO_LARGE: return "problem larger than the fixed scratch of this allocation-free entry point";
   }
   return "unknown status";
 }

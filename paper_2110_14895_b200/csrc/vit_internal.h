@@ -83,6 +83,11 @@ cudaError_t launch_head(const void* tokens, const float* g, const float* b, floa
                         const void* W, const float* bias, float* feat_scratch, float* logits,
                         int images, int T, int H, int classes, bool act_bf16, cudaStream_t s);
 
+// head with the feature scratch in a fixed device array of VIT_HEAD_STATIC_MAX_FLOATS floats
+cudaError_t launch_head_static(const void* tokens, const float* g, const float* b, float eps,
+                               const void* W, const float* bias, float* logits, int images, int T,
+                               int H, int classes, bool act_bf16, cudaStream_t s);
+
 bool tc_gemm_init();   // resolves the driver's tensor-map encoder; false if unavailable
 
 }  // namespace vit

@@ -34,8 +34,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
-template <int D>
-__global__ void __launch_bounds__(512, 1)
+template <int D, int NT, int MINB>
+__global__ void __launch_bounds__(NT, MINB)
 attention_bf16_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ out, int T, int heads) {
   constexpr int LD = D + 8;            // padded row (elements): keeps ldmatrix conflict-free
   constexpr int KS = D / 16;           // k-steps of QK^T
@@ -173,24 +173,32 @@ attention_bf16_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ out, int 
   }
 }
 
+template <int D, int NT, int MINB>
+cudaError_t launch_variant(const bf16* qkv, bf16* out, int images, int T, int heads, int nw, size_t smem,
+                           cudaStream_t s) {
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(attention_bf16_kernel<D, NT, MINB>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  attention_bf16_kernel<D, NT, MINB><<<images * heads, nw * 32, smem, s>>>(qkv, out, T, heads);
+  return cudaGetLastError();
+}
+
 template <int D>
 cudaError_t launch_d(const bf16* qkv, bf16* out, int images, int T, int heads, cudaStream_t s) {
   const int Tp = (T + 31) & ~31;
   const size_t smem = (size_t)2 * Tp * (D + 8) * sizeof(bf16);
   if (smem > 227 * 1024) return cudaErrorInvalidValue;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(attention_bf16_kernel<D>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
   const int ntiles = (T + 15) / 16;
   int nw = (ntiles + 1) / 2;
   if (nw < 1) nw = 1;
   if (nw > 16) nw = 16;
-  attention_bf16_kernel<D><<<images * heads, nw * 32, smem, s>>>(qkv, out, T, heads);
-  return cudaGetLastError();
+  // up to 9 warps: registers capped so that two CTAs share an SM
+  if (nw <= 9) return launch_variant<D, 288, 2>(qkv, out, images, T, heads, nw, smem, s);
+  return launch_variant<D, 512, 1>(qkv, out, images, T, heads, nw, smem, s);
 }
 
 }  // namespace

@@ -35,24 +35,20 @@ layernorm_bf16_kernel(const bf16* __restrict__ x, const float* __restrict__ g,
   if (row >= rows) return;
   const int nvec = cols >> 3;
   const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)row * cols);
-  float v[NCH][8];
-  float sum = 0.f;
+  uint4 u[NCH];                       // the row stays packed (bf16) in registers between passes
 #pragma unroll
   for (int i = 0; i < NCH; ++i) {
     const int idx = lane + 32 * i;
-    if (idx < nvec) {
-      const uint4 u = __ldg(xr + idx);
-      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+    u[i] = idx < nvec ? __ldg(xr + idx) : make_uint4(0, 0, 0, 0);
+  }
+  float sum = 0.f;
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float2 f = __bfloat1622float2(h[e]);
-        v[i][2 * e] = f.x;
-        v[i][2 * e + 1] = f.y;
-        sum += f.x + f.y;
-      }
-    } else {
+  for (int i = 0; i < NCH; ++i) {
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u[i]);
 #pragma unroll
-      for (int e = 0; e < 8; ++e) v[i][e] = 0.f;
+    for (int e = 0; e < 4; ++e) {
+      const float2 f = __bfloat1622float2(h[e]);
+      sum += f.x + f.y;               // padded chunks are zero
     }
   }
   const float mean = warp_sum(sum) / (float)cols;
@@ -60,10 +56,12 @@ layernorm_bf16_kernel(const bf16* __restrict__ x, const float* __restrict__ g,
 #pragma unroll
   for (int i = 0; i < NCH; ++i) {
     if (lane + 32 * i < nvec) {
+      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u[i]);
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const float c = v[i][e] - mean;
-        sq += c * c;
+      for (int e = 0; e < 4; ++e) {
+        const float2 f = __bfloat1622float2(h[e]);
+        const float c0 = f.x - mean, c1 = f.y - mean;
+        sq += c0 * c0 + c1 * c1;
       }
     }
   }
@@ -79,13 +77,15 @@ layernorm_bf16_kernel(const bf16* __restrict__ x, const float* __restrict__ g,
       const float4 b1 = __ldg(reinterpret_cast<const float4*>(b) + 2 * idx + 1);
       const float gg[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
       const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u[i]);
       uint4 o;
-      __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&o);
+      __nv_bfloat162* ho = reinterpret_cast<__nv_bfloat162*>(&o);
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        const float r0 = (v[i][2 * e] - mean) * rstd * gg[2 * e] + bb[2 * e];
-        const float r1 = (v[i][2 * e + 1] - mean) * rstd * gg[2 * e + 1] + bb[2 * e + 1];
-        h[e] = __floats2bfloat162_rn(r0, r1);
+        const float2 f = __bfloat1622float2(h[e]);
+        const float r0 = (f.x - mean) * rstd * gg[2 * e] + bb[2 * e];
+        const float r1 = (f.y - mean) * rstd * gg[2 * e + 1] + bb[2 * e + 1];
+        ho[e] = __floats2bfloat162_rn(r0, r1);
       }
       yr[idx] = o;
     }
@@ -363,22 +363,35 @@ __global__ void head_ln_kernel(const TIn* __restrict__ tokens, const float* __re
     feat[(size_t)img * H + i] = ((float)xr[i] - mean) * rstd * g[i] + b[i];
 }
 
+// One warp per class and group of HEAD_IMGS images: a weight element is loaded once and used
+// for every image of the group, and the groups give the grid enough warps to hide latency.
+constexpr int HEAD_IMGS = 8;
 template <typename TW>
 __global__ void __launch_bounds__(256)
 head_logits_kernel(const float* __restrict__ feat, const TW* __restrict__ W,
                    const float* __restrict__ bias, float* __restrict__ logits, int images, int H,
                    int classes) {
-  const int c = (int)((blockIdx.x * (size_t)blockDim.x + threadIdx.x) >> 5);
+  const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
+  const int img0 = blockIdx.y * HEAD_IMGS;
   if (c >= classes) return;
   const TW* wr = W + (size_t)c * H;
+  float acc[HEAD_IMGS];
+#pragma unroll
+  for (int j = 0; j < HEAD_IMGS; ++j) acc[j] = 0.f;
+  for (int i = lane; i < H; i += 32) {
+    const float w = (float)wr[i];
+#pragma unroll
+    for (int j = 0; j < HEAD_IMGS; ++j) {
+      const int img = img0 + j < images ? img0 + j : images - 1;
+      acc[j] = fmaf(feat[(size_t)img * H + i], w, acc[j]);
+    }
+  }
   const float bc = bias[c];
-  for (int img = 0; img < images; ++img) {
-    const float* f = feat + (size_t)img * H;
-    float s = 0.f;
-    for (int i = lane; i < H; i += 32) s = fmaf(f[i], (float)wr[i], s);
-    s = warp_sum(s);
-    if (lane == 0) logits[(size_t)img * classes + c] = s + bc;
+#pragma unroll
+  for (int j = 0; j < HEAD_IMGS; ++j) {
+    const float s = warp_sum(acc[j]);
+    if (lane == 0 && img0 + j < images) logits[(size_t)(img0 + j) * classes + c] = s + bc;
   }
 }
 
@@ -388,7 +401,7 @@ cudaError_t launch_head(const void* tokens, const float* g, const float* b, floa
   if (images <= 0) return cudaSuccess;
   const int threads = 256;
   const unsigned b1 = (unsigned)(((size_t)images * 32 + threads - 1) / threads);
-  const unsigned b2 = (unsigned)(((size_t)classes * 32 + threads - 1) / threads);
+  const dim3 b2((unsigned)((classes + 7) / 8), (unsigned)((images + HEAD_IMGS - 1) / HEAD_IMGS));
   if (act_bf16) {
     head_ln_kernel<bf16><<<b1, threads, 0, s>>>((const bf16*)tokens, g, b, eps, feat, images, T, H);
     head_logits_kernel<bf16><<<b2, threads, 0, s>>>(feat, (const bf16*)W, bias, logits, images, H, classes);

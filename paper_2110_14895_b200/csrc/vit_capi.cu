@@ -402,7 +402,7 @@ int vit_run_stage(vit_handle* h, int layer_begin, int layer_end, int mb, const v
     a.epilogue = EPI_BIAS; a.out = wide; a.ldo = (int)(3 * H);
     if ((st = linear(h, VIT_PROF_QKV, a, s)) != VIT_OK) return st;
     // y = attention(qkv)
-    if (b16) VIT_LAUNCH(h, VIT_PROF_ATTENTION, launch_attention_bf16((const bf16*)wide, (bf16*)y, mb, h->T, c.heads, h->d, s));
+    if (b16) VIT_LAUNCH(h, VIT_PROF_ATTENTION, launch_attention_bf16((const bf16*)wide, (bf16*)y, mb, h->T, c.heads, h->d, h->dev_status, s));
     else VIT_LAUNCH(h, VIT_PROF_ATTENTION, launch_attention_f32((const float*)wide, (float*)y, mb, h->T, c.heads, h->d, s));
     // x = x + y Wo^T + bo
     a = LinearArgs{};
@@ -559,7 +559,7 @@ int vit_op_attention(vit_handle* h, int dtype, int images, int T, int heads, int
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (dtype == VIT_BF16) {
     if (d % 16 || d > 128) return VIT_ERR_INVALID_ARG;
-    VIT_LAUNCH(h, VIT_PROF_ATTENTION, launch_attention_bf16((const bf16*)qkv, (bf16*)out, images, T, heads, d, s));
+    VIT_LAUNCH(h, VIT_PROF_ATTENTION, launch_attention_bf16((const bf16*)qkv, (bf16*)out, images, T, heads, d, h->dev_status, s));
   } else if (dtype == VIT_FP32) {
     VIT_LAUNCH(h, VIT_PROF_ATTENTION, launch_attention_f32((const float*)qkv, (float*)out, images, T, heads, d, s));
   } else {

@@ -66,8 +66,12 @@ struct Handle {
 cudaError_t launch_layernorm_bf16(const bf16* x, const float* g, const float* b, float eps,
                                   bf16* y, int rows, int cols, cudaStream_t s);
 cudaError_t launch_linear_tc(const LinearArgs& a, int* dev_status, cudaStream_t s);   // tcgen05 GEMM
+// attention: the tcgen05 kernel where it supports the shape, else the warp-level mma kernel
 cudaError_t launch_attention_bf16(const bf16* qkv, bf16* out, int images, int T, int heads, int d,
-                                  cudaStream_t s);
+                                  int* dev_status, cudaStream_t s);
+bool attention_tc_supported(int T, int d);
+cudaError_t launch_attention_tc(const bf16* qkv, bf16* out, int images, int T, int heads, int d,
+                                int* dev_status, cudaStream_t s);
 // fp32 family (SIMT)
 cudaError_t launch_layernorm_f32(const float* x, const float* g, const float* b, float eps,
                                  float* y, int rows, int cols, cudaStream_t s);

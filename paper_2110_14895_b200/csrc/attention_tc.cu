@@ -6,13 +6,16 @@
 // (d = 80 only) as 32-byte-swizzled rows.  The same tiles serve as K-major operands (Q, K in
 // S = Q K^T) and as the N-major operand (V in O = P V).  Per query tile:
 //   S = Q K^T        tcgen05.mma, 128 x NK x d, accumulator in tensor memory (NK fp32 columns)
-//   softmax          4 warps, one thread per query row: row max, exp2, row sum; P is written
-//                    back over S as packed bf16 (tcgen05.st), so scores never leave the SM
-//   O = P V          tcgen05.mma with A = P from tensor memory, B = V from shared memory
+//   softmax          8 warps, two threads per query row (each half of the keys): row max, exp2,
+//                    row sum, halves combined through shared memory; P is written back over S
+//                    as packed bf16 (tcgen05.st), so scores never leave the SM
+//   O = P V          tcgen05.mma with A = P from tensor memory, B = V from shared memory (for
+//                    d = 80, V is held as five 32-byte-swizzled blocks of 16 columns)
 //   epilogue         O / rowsum -> bf16 -> global
 // Keys beyond NK = 256 (the 257th token) are handled by the row's thread with plain FMAs on
 // copies of those K/V rows in shared memory.
-// Warps: 0-3 softmax/epilogue, 4 = TMA + MMA issue + tensor-memory allocation.
+// Warps: 0-7 softmax/epilogue (warp w reads tensor-memory lanes 32 (w % 4) ...), 8 = TMA + MMA
+// issue + tensor-memory allocation.
 // The two resident CTAs overlap one's softmax with the other's loads and MMAs.
 // Every mbarrier wait is bounded; on expiry the CTA raises the device status word and leaves.
 #include "vit_internal.h"
@@ -27,10 +30,11 @@ namespace {
 using namespace ptx;
 
 constexpr int QT = 128;          // queries per tile = tensor-memory lanes
-constexpr int MAX_EXTRA = 8;     // keys beyond NK handled without the tensor cores
-constexpr int NUM_THREADS = 5 * 32;
+constexpr int MAX_EXTRA = 4;     // keys beyond NK handled without the tensor cores
+constexpr int SOFTMAX_THREADS = 8 * 32;
+constexpr int NUM_THREADS = SOFTMAX_THREADS + 32;
+constexpr int MMA_WARP = 8;
 constexpr uint32_t TMEM_COLS = 256;
-constexpr uint32_t O_COL = 128;  // O accumulator columns [128, 128 + d); P occupies [0, NK / 2)
 
 // Shared-memory matrix descriptors for TMA-written tiles whose rows are one swizzle span wide
 // (128 or 32 bytes); groups of 8 rows are 8 spans apart.  The same descriptor form serves a
@@ -42,6 +46,11 @@ __device__ __forceinline__ uint64_t make_desc_sw128(uint32_t saddr) {
 __device__ __forceinline__ uint64_t make_desc_sw32(uint32_t saddr) {
   return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(256 >> 4) << 32) |
          ((uint64_t)1 << 46) | ((uint64_t)6 << 61);
+}
+// N-major operand made of several 32-byte-wide swizzled column blocks `lbo` bytes apart
+__device__ __forceinline__ uint64_t make_desc_sw32_blocks(uint32_t saddr, uint32_t lbo) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16) |
+         ((uint64_t)(256 >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)6 << 61);
 }
 __host__ __device__ constexpr uint32_t idesc_bf16(int n, bool b_n_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (b_n_major ? (1u << 16) : 0u) | ((uint32_t)(n >> 3) << 17) |
@@ -71,18 +80,42 @@ __device__ __forceinline__ float dot8(const uint4& a, const uint4& b, float acc)
 
 struct AttnMaps { CUtensorMap q64, q16, kv64, kv16; };
 
+// Tensor-memory columns (256 per CTA).  S occupies [0, NK).  The two threads of a row each own
+// half of the keys and overwrite S with P (bf16 pairs) only inside columns they have already
+// consumed themselves: half 0 walks its 32-key chunks upwards and packs P from column 0; half 1
+// walks its chunks downwards and packs P downwards from column NK.  O sits in between.
+template <int NK>
+struct TmemMap {
+  static constexpr int SPLIT = (NK / 64) * 32;              // keys [0, SPLIT) -> half 0, [SPLIT, NK) -> half 1
+  static constexpr int END1 = SPLIT + ((NK - SPLIT + 31) / 32) * 32;   // end of half 1's last (maybe partial) chunk
+  static constexpr uint32_t O_COL = SPLIT / 2;
+  // first P column of the 32-key chunk that starts at key c0
+  __host__ __device__ static constexpr uint32_t p_col(int c0) {
+    return c0 < SPLIT ? (uint32_t)(c0 / 2) : (uint32_t)(NK - 16 * ((END1 - 32 - c0) / 32 + 1));
+  }
+  // P columns of the 16 keys of MMA step ks
+  __host__ __device__ static constexpr uint32_t p_col_step(int ks) {
+    return 16 * ks < SPLIT ? (uint32_t)(8 * ks)
+                           : p_col(SPLIT + ((16 * ks - SPLIT) / 32) * 32) + (uint32_t)((((16 * ks - SPLIT) / 16) % 2) * 8);
+  }
+};
+
 template <int D, int NK>
 struct Smem {
   static constexpr bool TAIL = D > 64;                 // columns [64, D) live in the 32-byte part
   static constexpr uint32_t KA = NK * 128, QA = QT * 128;
   static constexpr uint32_t KB = TAIL ? NK * 32 : 0, QB = TAIL ? QT * 32 : 0;
-  static constexpr uint32_t OFF_KA = 0, OFF_VA = KA, OFF_QA = 2 * KA;
-  static constexpr uint32_t OFF_KB = 2 * KA + QA, OFF_VB = OFF_KB + KB, OFF_QB = OFF_VB + KB;
+  static constexpr uint32_t VBYTES = NK * D * 2;       // D = 64: one 128-byte-swizzled tile;
+                                                       // D = 80: five 32-byte-swizzled 16-column blocks
+  static constexpr uint32_t OFF_KA = 0, OFF_QA = KA, OFF_V = KA + QA;
+  static constexpr uint32_t OFF_KB = OFF_V + VBYTES, OFF_QB = OFF_KB + KB;
   static constexpr uint32_t OFF_XK = OFF_QB + QB;      // extra K rows, plain [MAX_EXTRA][D]
   static constexpr uint32_t OFF_XV = OFF_XK + MAX_EXTRA * D * 2;
-  static constexpr uint32_t OFF_BARS = OFF_XV + MAX_EXTRA * D * 2;
+  static constexpr uint32_t OFF_RED = OFF_XV + MAX_EXTRA * D * 2;   // float [2 halves][QT] row max, then [2][QT] row sum
+  static constexpr uint32_t OFF_SX = OFF_RED + 4 * QT * 4;          // float [2 tiles][MAX_EXTRA][QT] extra-key scores
+  static constexpr uint32_t OFF_BARS = OFF_SX + 2 * MAX_EXTRA * QT * 4;
   static constexpr uint32_t BYTES = OFF_BARS + 128 + 1024 /*alignment slack*/;
-  static constexpr uint32_t KV_TX = 2 * (KA + KB), Q_TX = QA + QB;
+  static constexpr uint32_t KV_TX = KA + KB + VBYTES, Q_TX = QA + QB;
 };
 
 template <int D, int NK>
@@ -98,9 +131,9 @@ attention_tc_kernel(const __grid_constant__ AttnMaps maps, const bf16* __restric
   const uint32_t kv_full = smem_u32(&bars[0]);   // K, V landed                 (TMA bytes)
   const uint32_t q_full = smem_u32(&bars[1]);    // Q tile landed               (TMA bytes)
   const uint32_t s_ready = smem_u32(&bars[2]);   // S complete in tensor memory (MMA commit)
-  const uint32_t p_ready = smem_u32(&bars[3]);   // P written                   (128 arrivals)
+  const uint32_t p_ready = smem_u32(&bars[3]);   // P written                   (256 arrivals)
   const uint32_t o_ready = smem_u32(&bars[4]);   // O complete                  (MMA commit)
-  const uint32_t t_free = smem_u32(&bars[5]);    // O read, tensor memory free  (128 arrivals)
+  const uint32_t t_free = smem_u32(&bars[5]);    // O read, tensor memory free  (256 arrivals)
   const uint32_t q_read = smem_u32(&bars[6]);    // Q rows read by their threads (128 arrivals)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(&bars[7]);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -118,13 +151,13 @@ attention_tc_kernel(const __grid_constant__ AttnMaps maps, const bf16* __restric
     mbar_init(kv_full, 1);
     mbar_init(q_full, 1);
     mbar_init(s_ready, 1);
-    mbar_init(p_ready, QT);
+    mbar_init(p_ready, SOFTMAX_THREADS);
     mbar_init(o_ready, 1);
-    mbar_init(t_free, QT);
+    mbar_init(t_free, SOFTMAX_THREADS);
     mbar_init(q_read, QT);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 4) tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+  if (warp == MMA_WARP) tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
   // copies of the K and V rows of the keys beyond NK, as plain rows
   for (int i = threadIdx.x; i < n_extra * CH * 2; i += NUM_THREADS) {
     const int which = i / (n_extra * CH), j = i % (n_extra * CH), e = j / CH, c = j % CH;
@@ -136,17 +169,20 @@ attention_tc_kernel(const __grid_constant__ AttnMaps maps, const bf16* __restric
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == 4) {
+  if (warp == MMA_WARP) {
     // ------------------------------------------------------------------ TMA + MMA issuer
     if (lane == 0) {
       const int row_g = img * T;                 // global row of token 0
       const int col_q = hd * D, col_k = H + hd * D, col_v = 2 * H + hd * D;
       mbar_arrive_expect_tx(kv_full, L::KV_TX);
       tma_load_2d(sb + L::OFF_KA, &maps.kv64, col_k, row_g, kv_full);
-      tma_load_2d(sb + L::OFF_VA, &maps.kv64, col_v, row_g, kv_full);
       if (L::TAIL) {
         tma_load_2d(sb + L::OFF_KB, &maps.kv16, col_k + 64, row_g, kv_full);
-        tma_load_2d(sb + L::OFF_VB, &maps.kv16, col_v + 64, row_g, kv_full);
+#pragma unroll
+        for (int a = 0; a < D / 16; ++a)
+          tma_load_2d(sb + L::OFF_V + (uint32_t)(a * NK * 32), &maps.kv16, col_v + 16 * a, row_g, kv_full);
+      } else {
+        tma_load_2d(sb + L::OFF_V, &maps.kv64, col_v, row_g, kv_full);
       }
       mbar_arrive_expect_tx(q_full, L::Q_TX);
       tma_load_2d(sb + L::OFF_QA, &maps.q64, col_q, row_g, q_full);
@@ -180,97 +216,120 @@ attention_tc_kernel(const __grid_constant__ AttnMaps maps, const bf16* __restric
         tc_fence_after();
         // O = P V: A = P in tensor memory (8 columns per 16 keys); B = V, 16 keys per step =
         // two 8-row groups of the tile
-#pragma unroll 4
+#pragma unroll
         for (int k = 0; k < NK / 16; ++k) {
-          umma_bf16_ts(tmem_base + O_COL, tmem_base + (uint32_t)(k * 8),
-                       make_desc_sw128(sb + L::OFF_VA + (uint32_t)(k * 2048)), idesc_bf16(64, true),
-                       k > 0 ? 1u : 0u);
-          if (L::TAIL)
-            umma_bf16_ts(tmem_base + O_COL + 64, tmem_base + (uint32_t)(k * 8),
-                         make_desc_sw32(sb + L::OFF_VB + (uint32_t)(k * 512)), idesc_bf16(D - 64, true),
-                         k > 0 ? 1u : 0u);
+          const uint64_t bdesc = L::TAIL ? make_desc_sw32_blocks(sb + L::OFF_V + (uint32_t)(k * 512), NK * 32)
+                                         : make_desc_sw128(sb + L::OFF_V + (uint32_t)(k * 2048));
+          umma_bf16_ts(tmem_base + TmemMap<NK>::O_COL, tmem_base + TmemMap<NK>::p_col_step(k), bdesc,
+                       idesc_bf16(D, true), k > 0 ? 1u : 0u);
         }
         umma_commit(o_ready);
       }
     }
   } else {
     // ------------------------------------------------------------------ softmax + epilogue
-    const int row = warp * 32 + lane;                       // tensor-memory lane
-    const uint32_t lane_addr = tmem_base + ((uint32_t)(warp * 32) << 16);
+    const int quarter = warp & 3, half = warp >> 2;
+    const int row = quarter * 32 + lane;                    // tensor-memory lane = query row of the tile
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
     const float sl2 = 1.4426950408889634f / sqrtf((float)D);   // log2(e) / sqrt(d)
+    using TM = TmemMap<NK>;
+    constexpr int SPLIT = TM::SPLIT;
+    constexpr uint32_t O_COL = TM::O_COL;
+    const int k_begin = half ? SPLIT : 0, k_end = half ? NK : SPLIT;
+    float* red = reinterpret_cast<float*>(smem + L::OFF_RED);     // [0..1][QT] max, [2..3][QT] sum
+    float* sx = reinterpret_cast<float*>(smem + L::OFF_SX);       // [tile & 1][MAX_EXTRA][QT]
+    auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(1 + quarter) : "memory"); };
     bool ok = true;
-    for (int t = 0; t < ntiles && ok; ++t) {
-      const uint32_t ph = (uint32_t)(t & 1);
-      const int tok = t * QT + row;
-      const bool valid = tok < T;
-      const bool warp_active = t * QT + warp * 32 < T;      // any valid row in this warp
-      // scores of the keys beyond NK, by hand (fp32 accumulation of bf16 products)
-      float s_ex[MAX_EXTRA];
+
+    // Scores of the keys beyond NK for tile `tt` (half 0 only), by hand: the row of Q is read back
+    // from the swizzled tile, the K rows are plain copies.  Results go to shared memory for both
+    // halves; arrives on q_read.
+    auto extra_scores = [&](int tt) -> bool {
+      if (n_extra == 0 || half != 0) return true;
+      if (!mbar_wait(q_full, (uint32_t)(tt & 1), abort_flag)) return false;
+      if (tt * QT + quarter * 32 < T) {
+        uint4 q[CH];
 #pragma unroll
-      for (int e = 0; e < MAX_EXTRA; ++e) s_ex[e] = -INFINITY;
-      if (n_extra > 0) {
-        if (!mbar_wait(q_full, ph, abort_flag)) { ok = false; break; }
-        if (warp_active) {
-          uint4 q[CH];
+        for (int c = 0; c < 8; ++c) q[c] = lds128(sb + L::OFF_QA + (uint32_t)(row * 128 + ((c ^ (row & 7)) << 4)));
 #pragma unroll
-          for (int c = 0; c < 8; ++c) q[c] = lds128(sb + L::OFF_QA + (uint32_t)(row * 128 + ((c ^ (row & 7)) << 4)));
+        for (int c = 8; c < CH; ++c)
+          q[c] = lds128(sb + L::OFF_QB + (uint32_t)(row * 32 + (((c - 8) ^ ((row >> 2) & 1)) << 4)));
 #pragma unroll
-          for (int c = 8; c < CH; ++c)
-            q[c] = lds128(sb + L::OFF_QB + (uint32_t)(row * 32 + (((c - 8) ^ ((row >> 2) & 1)) << 4)));
+        for (int e = 0; e < MAX_EXTRA; ++e) {
+          if (e < n_extra) {
+            float acc = 0.f;
 #pragma unroll
-          for (int e = 0; e < MAX_EXTRA; ++e) {
-            if (e < n_extra) {
-              float acc = 0.f;
-#pragma unroll
-              for (int c = 0; c < CH; ++c) acc = dot8(q[c], lds128(sb + L::OFF_XK + (uint32_t)((e * CH + c) * 16)), acc);
-              s_ex[e] = acc;
-            }
+            for (int c = 0; c < CH; ++c) acc = dot8(q[c], lds128(sb + L::OFF_XK + (uint32_t)((e * CH + c) * 16)), acc);
+            sx[((tt & 1) * MAX_EXTRA + e) * QT + row] = acc;
           }
         }
-        mbar_arrive(q_read);
       }
+      mbar_arrive(q_read);
+      return true;
+    };
+    ok = extra_scores(0);
+
+    for (int t = 0; t < ntiles && ok; ++t) {
+      const uint32_t ph = (uint32_t)(t & 1);
+      const bool warp_active = t * QT + quarter * 32 < T;   // any valid row in this warp
+      const float* sxt = sx + (t & 1) * MAX_EXTRA * QT;
       if (!mbar_wait(s_ready, ph, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      float l = 1.f;
-      float p_ex[MAX_EXTRA];
-#pragma unroll
-      for (int e = 0; e < MAX_EXTRA; ++e) p_ex[e] = 0.f;
+      float msl = 0.f;
       if (warp_active) {
-        // pass 1: row maximum
+        // pass 1: maximum over this half's keys
         float m = -INFINITY;
+        if (half == 0) {
 #pragma unroll
-        for (int e = 0; e < MAX_EXTRA; ++e) m = fmaxf(m, s_ex[e]);
+          for (int e = 0; e < MAX_EXTRA; ++e)
+            if (e < n_extra) m = fmaxf(m, sxt[e * QT + row]);
+        }
 #pragma unroll 1
-        for (int c0 = 0; c0 < NK; c0 += 32) {
+        for (int c0 = k_begin; c0 < k_end; c0 += 32) {
           uint32_t r[32];
           tmem_ld32(lane_addr + (uint32_t)c0, r);      // the last chunk may run past NK: masked below
           tmem_ld_wait();
-          if (c0 + 32 <= T) {
+          if (c0 + 32 <= T && c0 + 32 <= NK) {
+            float m2[2] = {m, m};
 #pragma unroll
-            for (int j = 0; j < 32; ++j) m = fmaxf(m, __uint_as_float(r[j]));
+            for (int j = 0; j < 32; j += 4) {
+              asm("max.f32 %0, %0, %1, %2;" : "+f"(m2[0]) : "f"(__uint_as_float(r[j])), "f"(__uint_as_float(r[j + 1])));
+              asm("max.f32 %0, %0, %1, %2;" : "+f"(m2[1]) : "f"(__uint_as_float(r[j + 2])), "f"(__uint_as_float(r[j + 3])));
+            }
+            m = fmaxf(m2[0], m2[1]);
           } else {
 #pragma unroll
             for (int j = 0; j < 32; ++j)
               if (c0 + j < T && c0 + j < NK) m = fmaxf(m, __uint_as_float(r[j]));
           }
         }
-        // pass 2: p = exp2((s - m) * sl2), row sum, P (bf16) back into tensor memory
-        const float msl = m * sl2;
-        l = 0.f;
+        red[half * QT + row] = m;
+      }
+      pair_sync();
+      float l = 0.f;
+      if (warp_active) {
+        msl = fmaxf(red[row], red[QT + row]) * sl2;
+        // pass 2: p = exp2((s - m) * sl2), partial row sum, P (bf16) back into tensor memory
+        // (half 0 upwards, half 1 downwards: see TmemMap)
+        const int nchunks = (k_end - k_begin + 31) / 32;
 #pragma unroll 1
-        for (int c0 = 0; c0 < NK; c0 += 32) {
+        for (int i = 0; i < nchunks; ++i) {
+          const int c0 = half ? k_begin + 32 * (nchunks - 1 - i) : k_begin + 32 * i;
           uint32_t r[32];
           tmem_ld32(lane_addr + (uint32_t)c0, r);
           tmem_ld_wait();
           uint32_t pk[16];
-          if (c0 + 32 <= T) {
+          if (c0 + 32 <= T && c0 + 32 <= NK) {
+            float l2[2] = {0.f, 0.f};
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
               const float p0 = ex2_approx(fmaf(__uint_as_float(r[2 * j]), sl2, -msl));
               const float p1 = ex2_approx(fmaf(__uint_as_float(r[2 * j + 1]), sl2, -msl));
-              l += p0 + p1;
+              l2[0] += p0;
+              l2[1] += p1;
               pk[j] = pack_bf16(p0, p1);
             }
+            l += l2[0] + l2[1];
           } else {
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
@@ -281,66 +340,76 @@ attention_tc_kernel(const __grid_constant__ AttnMaps maps, const bf16* __restric
               pk[j] = pack_bf16(p0, p1);
             }
           }
-          tmem_st16(lane_addr + (uint32_t)(c0 >> 1), pk);
+          tmem_st16(lane_addr + TM::p_col(c0), pk);
         }
-#pragma unroll
-        for (int e = 0; e < MAX_EXTRA; ++e) {
-          if (e < n_extra) {
-            p_ex[e] = ex2_approx(fmaf(s_ex[e], sl2, -msl));
-            l += p_ex[e];
-          }
-        }
+        red[(2 + half) * QT + row] = l;
         tmem_st_wait();
       }
       tc_fence_before();
       mbar_arrive(p_ready);
-      // epilogue: O / l (+ the hand-computed keys' share) -> bf16 -> global
+      // while the tensor core runs P V: the extra keys' scores of the next tile
+      if (t + 1 < ntiles && !extra_scores(t + 1)) { ok = false; break; }
+      // epilogue: O (+ the hand-computed keys' share) / l -> bf16 -> global; this half's columns
       if (!mbar_wait(o_ready, ph, abort_flag)) { ok = false; break; }
       tc_fence_after();
+      pair_sync();                                          // both partial sums are in shared memory
+      constexpr int G0 = (D / 16 + 1) / 2;                  // 16-column groups [0, G0) -> half 0, the rest -> half 1
+      const int g_begin = half ? G0 : 0, g_end = half ? D / 16 : G0;
+      uint32_t oreg[G0 * 16];
       if (warp_active) {
+#pragma unroll
+        for (int g = 0; g < G0; ++g)
+          if (g_begin + g < g_end)
+            tmem_ld16(lane_addr + O_COL + (uint32_t)((g_begin + g) * 16), *reinterpret_cast<uint32_t(*)[16]>(&oreg[g * 16]));
+        tmem_ld_wait();
+      }
+      tc_fence_before();
+      mbar_arrive(t_free);               // the next tile's S may overwrite tensor memory now
+      const int tok = t * QT + row;
+      if (warp_active && tok < T) {
+        l = red[2 * QT + row] + red[3 * QT + row];
+        float p_ex[MAX_EXTRA];
+#pragma unroll
+        for (int e = 0; e < MAX_EXTRA; ++e) {
+          p_ex[e] = e < n_extra ? ex2_approx(fmaf(sxt[e * QT + row], sl2, -msl)) : 0.f;
+          l += p_ex[e];
+        }
         const float inv = 1.0f / l;
-        uint4* orow = reinterpret_cast<uint4*>(out + ((size_t)img * T + (valid ? tok : 0)) * H + (size_t)hd * D);
+        uint4* orow = reinterpret_cast<uint4*>(out + ((size_t)img * T + tok) * H + (size_t)hd * D);
 #pragma unroll
-        for (int c = 0; c < D / 16; ++c) {
-          uint32_t r[16];
-          tmem_ld16(lane_addr + O_COL + (uint32_t)(c * 16), r);
-          tmem_ld_wait();
-          float o[16];
+        for (int g = 0; g < G0; ++g) {
+          if (g_begin + g < g_end) {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) o[j] = __uint_as_float(r[j]);
-          if (n_extra > 0) {
+            for (int q = 0; q < 2; ++q) {
+              const int c = (g_begin + g) * 2 + q;         // 16-byte chunk of the row
+              float o[8];
 #pragma unroll
-            for (int e = 0; e < MAX_EXTRA; ++e) {
-              if (e < n_extra) {
+              for (int j = 0; j < 8; ++j) o[j] = __uint_as_float(oreg[g * 16 + q * 8 + j]);
+              if (n_extra > 0) {
 #pragma unroll
-                for (int q = 0; q < 2; ++q) {
-                  const uint4 va = lds128(sb + L::OFF_XV + (uint32_t)((e * CH + 2 * c + q) * 16));
-                  const __nv_bfloat162* vh = reinterpret_cast<const __nv_bfloat162*>(&va);
+                for (int e = 0; e < MAX_EXTRA; ++e) {
+                  if (e < n_extra) {
+                    const uint4 va = lds128(sb + L::OFF_XV + (uint32_t)((e * CH + c) * 16));
+                    const __nv_bfloat162* vh = reinterpret_cast<const __nv_bfloat162*>(&va);
 #pragma unroll
-                  for (int j = 0; j < 4; ++j) {
-                    const float2 v2 = __bfloat1622float2(vh[j]);
-                    o[q * 8 + 2 * j] = fmaf(p_ex[e], v2.x, o[q * 8 + 2 * j]);
-                    o[q * 8 + 2 * j + 1] = fmaf(p_ex[e], v2.y, o[q * 8 + 2 * j + 1]);
+                    for (int j = 0; j < 4; ++j) {
+                      const float2 v2 = __bfloat1622float2(vh[j]);
+                      o[2 * j] = fmaf(p_ex[e], v2.x, o[2 * j]);
+                      o[2 * j + 1] = fmaf(p_ex[e], v2.y, o[2 * j + 1]);
+                    }
                   }
                 }
               }
-            }
-          }
-          if (valid) {
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
               uint4 w;
-              w.x = pack_bf16(o[q * 8 + 0] * inv, o[q * 8 + 1] * inv);
-              w.y = pack_bf16(o[q * 8 + 2] * inv, o[q * 8 + 3] * inv);
-              w.z = pack_bf16(o[q * 8 + 4] * inv, o[q * 8 + 5] * inv);
-              w.w = pack_bf16(o[q * 8 + 6] * inv, o[q * 8 + 7] * inv);
-              orow[2 * c + q] = w;
+              w.x = pack_bf16(o[0] * inv, o[1] * inv);
+              w.y = pack_bf16(o[2] * inv, o[3] * inv);
+              w.z = pack_bf16(o[4] * inv, o[5] * inv);
+              w.w = pack_bf16(o[6] * inv, o[7] * inv);
+              orow[c] = w;
             }
           }
         }
       }
-      tc_fence_before();
-      mbar_arrive(t_free);
     }
   }
 
@@ -351,7 +420,7 @@ attention_tc_kernel(const __grid_constant__ AttnMaps maps, const bf16* __restric
   __syncthreads();
   tc_fence_after();
   if (threadIdx.x == 0 && *abort_flag) atomicExch(dev_status, (int)VIT_ERR_TIMEOUT);
-  if (warp == 4) {
+  if (warp == MMA_WARP) {
     __syncwarp();
     tmem_dealloc(tmem_base, TMEM_COLS);
   }

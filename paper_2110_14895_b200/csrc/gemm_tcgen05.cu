@@ -58,20 +58,20 @@ template <int BN> __host__ __device__ constexpr uint32_t make_idesc() {
          | ((uint32_t)(BM >> 4) << 24);  // M / 16
 }
 
-// gelu(v) = 0.5 v (1 + erf(v / sqrt 2)) with erfc(z) = (a1 t + ... + a5 t^5) exp(-z^2),
-// t = 1 / (1 + p z), z >= 0 (Abramowitz & Stegun 7.1.26, |error| <= 1.5e-7), on the MUFU
-// reciprocal and exp2.  For v >= 0: v - 0.5 v erfc(z); for v < 0: 0.5 v erfc(z).
+// gelu(v) = 0.5 v (1 + erf(v / sqrt 2)) = max(v, 0) - 0.5 |v| erfc(|v| / sqrt 2), with
+// erfc(z) = (a1 t + ... + a5 t^5) exp(-z^2), t = 1 / (1 + p z), z >= 0 (Abramowitz & Stegun
+// 7.1.26, |error| <= 1.5e-7), on the MUFU reciprocal and exp2.  The factor 0.5 is folded into
+// the coefficients and 1/sqrt 2 into p and the exponent scale.
 __device__ __forceinline__ float gelu_erf(float v) {
-  const float z = fabsf(v) * 0.70710678118654752440f;
-  const float t = __fdividef(1.0f, fmaf(0.3275911f, z, 1.0f));
-  float e;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(z * z * -1.4426950408889634f));
-  float q = fmaf(1.061405429f, t, -1.453152027f);
-  q = fmaf(q, t, 1.421413741f);
-  q = fmaf(q, t, -0.284496736f);
-  q = fmaf(q, t, 0.254829592f);
-  const float h = 0.5f * v * (q * t * e);
-  return v >= 0.f ? v - h : h;
+  const float a = fabsf(v);
+  float t, e;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.3275911f * 0.70710678118654752440f, a, 1.0f)));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(a * a * (-0.5f * 1.4426950408889634f)));
+  float q = fmaf(0.5f * 1.061405429f, t, 0.5f * -1.453152027f);
+  q = fmaf(q, t, 0.5f * 1.421413741f);
+  q = fmaf(q, t, 0.5f * -0.284496736f);
+  q = fmaf(q, t, 0.5f * 0.254829592f);
+  return fmaxf(v, 0.f) - q * t * e * a;
 }
 
 struct TcParams {

@@ -8,11 +8,17 @@
 //               the same way, by TMA load), so global traffic is coalesced and asynchronous
 // Two accumulators live in tensor memory (2 x BN columns) so the epilogue of tile i overlaps the
 // main loop of tile i+1.  Tiles are handed out statically (tile = blockIdx.x + i * gridDim.x).
+// For large problems the kernel runs as CTA pairs (CTAS = 2, a cluster of two): one 256 x 256
+// tile per pair, each CTA loads its own 128 rows of a and half of the w tile (no multicast), the
+// even CTA issues tcgen05.mma.cta_group::2 for both, and each CTA drains its own 128 rows of the
+// accumulator.  Shared-memory fill traffic per flop drops by a third, which leaves room for the
+// output stores.
 // Every mbarrier wait is bounded; on expiry the CTA raises the device status word and leaves.
 #include "vit_internal.h"
 #include "sm100_ptx.cuh"
 
 #include <cuda.h>
+#include <cstdlib>
 
 namespace vit {
 
@@ -26,10 +32,11 @@ constexpr int UMMA_K = 16;
 constexpr int NUM_EPI_WARPS = 8;
 constexpr int NUM_THREADS = (2 + NUM_EPI_WARPS) * 32;
 
-template <int BN> struct Cfg {
-  static constexpr int STAGES = (BN == 256) ? 4 : 6;
+template <int BN, int CTAS> struct Cfg {
+  static constexpr int B_ROWS = BN / CTAS;                 // rows of the w tile this CTA loads
+  static constexpr int STAGES = (B_ROWS == 256) ? 4 : 6;
   static constexpr int A_BYTES = BM * BK * 2;
-  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int B_BYTES = B_ROWS * BK * 2;
   static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int TMEM_COLS = 2 * BN;                 // 512 or 256: a power of two
   static constexpr int STAGING_BYTES = NUM_EPI_WARPS * 4096;   // 32 rows x 128 B per epilogue warp
@@ -50,12 +57,12 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
 }
 
 // Instruction descriptor for kind::f16: fp32 accumulate, bf16 x bf16, both operands K-major.
-template <int BN> __host__ __device__ constexpr uint32_t make_idesc() {
+template <int BN, int CTAS> __host__ __device__ constexpr uint32_t make_idesc() {
   return (1u << 4)                       // D format: f32
          | (1u << 7)                     // A format: bf16
          | (1u << 10)                    // B format: bf16
          | ((uint32_t)(BN >> 3) << 17)   // N / 8
-         | ((uint32_t)(BM >> 4) << 24);  // M / 16
+         | ((uint32_t)((BM * CTAS) >> 4) << 24);  // M / 16 (256 rows across a CTA pair)
 }
 
 // gelu(v) = 0.5 v (1 + erf(v / sqrt 2)) = max(v, 0) - 0.5 |v| erfc(|v| / sqrt 2), with
@@ -86,12 +93,12 @@ struct TcParams {
   int* dev_status;
 };
 
-template <int BN, int EPI>
+template <int BN, int EPI, int CTAS>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w,
                  const __grid_constant__ CUtensorMap tm_out, const __grid_constant__ CUtensorMap tm_res,
                  const TcParams p) {
-  using C = Cfg<BN>;
+  using C = Cfg<BN, CTAS>;
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte alignment: the swizzle pattern and the descriptors assume it
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -109,6 +116,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_kb = (p.K + BK - 1) / BK;
   const int total_tiles = p.tiles_m * p.tiles_n;
+  // scheduling unit: a CTA, or a pair of CTAs working on one 256-row tile
+  const uint32_t rank = CTAS == 2 ? cluster_ctarank() : 0u;
+  const int unit = blockIdx.x / CTAS, num_units = gridDim.x / CTAS;
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
@@ -118,7 +128,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&tfull_bar[i]), 1);
-      mbar_init(smem_u32(&tempty_bar[i]), NUM_EPI_WARPS);
+      mbar_init(smem_u32(&tempty_bar[i]), NUM_EPI_WARPS * CTAS);
     }
     for (int i = 0; i < NUM_EPI_WARPS; ++i) mbar_init(smem_u32(&res_bar[i]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -127,14 +137,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_out)) : "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
-                     smem_u32(tmem_slot)),
-                 "r"((uint32_t)C::TMEM_COLS)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (CTAS == 2) tmem_alloc_pair(smem_u32(tmem_slot), (uint32_t)C::TMEM_COLS);
+    else tmem_alloc(smem_u32(tmem_slot), (uint32_t)C::TMEM_COLS);
   }
   tc_fence_before();
   __syncthreads();
+  if (CTAS == 2) cluster_sync();          // the peer's barriers are initialised before anyone signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -144,29 +152,38 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int m0 = (tile / p.tiles_n) * BM, n0 = (tile % p.tiles_n) * BN;
+      for (int tile = unit; tile < total_tiles && ok; tile += num_units) {
+        const int m0 = (tile / p.tiles_n) * (BM * CTAS) + (int)rank * BM;
+        const int n0 = (tile % p.tiles_n) * BN + (int)rank * C::B_ROWS;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1, abort_flag)) { ok = false; break; }
           const uint32_t fb = smem_u32(&full_bar[stage]);
-          mbar_arrive_expect_tx(fb, C::STAGE_BYTES);
           const uint32_t sa = smem_u32(tiles + stage * C::STAGE_BYTES);
-          tma_load_2d(sa, &tm_a, kb * BK, m0, fb);
-          tma_load_2d(sa + C::A_BYTES, &tm_w, kb * BK, n0, fb);
+          if (CTAS == 2) {
+            // both CTAs' copies are counted on the even CTA's barrier, which expects all the bytes
+            const uint32_t fb0 = map_to_cta(fb, 0);
+            if (rank == 0) mbar_arrive_expect_tx(fb, 2 * C::STAGE_BYTES);
+            tma_load_2d_pair(sa, &tm_a, kb * BK, m0, fb0);
+            tma_load_2d_pair(sa + C::A_BYTES, &tm_w, kb * BK, n0, fb0);
+          } else {
+            mbar_arrive_expect_tx(fb, C::STAGE_BYTES);
+            tma_load_2d(sa, &tm_a, kb * BK, m0, fb);
+            tma_load_2d(sa + C::A_BYTES, &tm_w, kb * BK, n0, fb);
+          }
           if (++stage == C::STAGES) { stage = 0; phase ^= 1; }
         }
       }
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc<BN>();
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = make_idesc<BN, CTAS>();
       int stage = 0;
       uint32_t phase = 0;
       int buf = 0;
       uint32_t aphase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      for (int tile = unit; tile < total_tiles && ok; tile += num_units) {
         if (!mbar_wait(smem_u32(&tempty_bar[buf]), aphase ^ 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
@@ -179,14 +196,21 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // advancing 16 elements along K = 32 bytes = 2 units of the encoded start address
-            umma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
-                      (kb > 0 || k > 0) ? 1u : 0u);
+            if (CTAS == 2)
+              umma_bf16_pair(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
+                             (kb > 0 || k > 0) ? 1u : 0u);
+            else
+              umma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
+                        (kb > 0 || k > 0) ? 1u : 0u);
           }
-          umma_commit(smem_u32(&empty_bar[stage]));   // frees the stage when these MMAs retire
+          // frees the stage (in both CTAs of a pair) when these MMAs retire
+          if (CTAS == 2) umma_commit_pair(smem_u32(&empty_bar[stage]));
+          else umma_commit(smem_u32(&empty_bar[stage]));
           if (++stage == C::STAGES) { stage = 0; phase ^= 1; }
         }
         if (!ok) break;
-        umma_commit(smem_u32(&tfull_bar[buf]));       // accumulator complete
+        if (CTAS == 2) umma_commit_pair(smem_u32(&tfull_bar[buf]));   // accumulator complete
+        else umma_commit(smem_u32(&tfull_bar[buf]));
         if (++buf == 2) { buf = 0; aphase ^= 1; }
       }
     }
@@ -200,8 +224,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     uint32_t aphase = 0;
     if (EPI == EPI_BIAS_POS) {
       // patch embedding: rows are scattered to token 1 + patch of their image, direct stores
-      for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-        const int m0 = (tile / p.tiles_n) * BM, n0 = (tile % p.tiles_n) * BN;
+      for (int tile = unit; tile < total_tiles; tile += num_units) {
+        const int m0 = (tile / p.tiles_n) * (BM * CTAS) + (int)rank * BM, n0 = (tile % p.tiles_n) * BN;
         if (!mbar_wait(smem_u32(&tfull_bar[buf]), aphase, abort_flag)) break;
         tc_fence_after();
         const int row = m0 + quarter * 32 + lane;
@@ -236,7 +260,11 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[buf]));
+        if (lane == 0) {
+          // the accumulator buffer is handed back to the MMA issuer (the even CTA of a pair)
+          if (CTAS == 2) mbar_arrive_cluster(map_to_cta(smem_u32(&tempty_bar[buf]), 0));
+          else mbar_arrive(smem_u32(&tempty_bar[buf]));
+        }
         if (++buf == 2) { buf = 0; aphase ^= 1; }
       }
     } else {
@@ -246,8 +274,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       const uint32_t rb = smem_u32(&res_bar[ew]);
       uint32_t rphase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const int m0 = (tile / p.tiles_n) * BM, n0 = (tile % p.tiles_n) * BN;
+      for (int tile = unit; tile < total_tiles && ok; tile += num_units) {
+        const int m0 = (tile / p.tiles_n) * (BM * CTAS) + (int)rank * BM, n0 = (tile % p.tiles_n) * BN;
         const int row0 = m0 + quarter * 32;
 #pragma unroll 1
         for (int cb = 0; cb < COLS_PER_WARP / 64; ++cb) {
@@ -325,7 +353,11 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         if (!ok) break;
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[buf]));
+        if (lane == 0) {
+          // the accumulator buffer is handed back to the MMA issuer (the even CTA of a pair)
+          if (CTAS == 2) mbar_arrive_cluster(map_to_cta(smem_u32(&tempty_bar[buf]), 0));
+          else mbar_arrive(smem_u32(&tempty_bar[buf]));
+        }
         if (++buf == 2) { buf = 0; aphase ^= 1; }
       }
       if (lane == 0) tma_store_wait_all();
@@ -337,13 +369,13 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
   if (*abort_flag) __nanosleep(200000);   // let copies and MMAs in flight land before leaving
   tc_fence_before();
   __syncthreads();
+  if (CTAS == 2) cluster_sync();          // neither CTA leaves while the other may still touch it
   tc_fence_after();
   if (threadIdx.x == 0 && *abort_flag) atomicExch(p.dev_status, (int)VIT_ERR_TIMEOUT);
   if (warp == 1) {
     __syncwarp();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
-                 "r"((uint32_t)C::TMEM_COLS)
-                 : "memory");
+    if (CTAS == 2) tmem_dealloc_pair(tmem_base, (uint32_t)C::TMEM_COLS);
+    else tmem_dealloc(tmem_base, (uint32_t)C::TMEM_COLS);
   }
 }
 
@@ -354,6 +386,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
 int g_num_sms = 0;
+int g_pair_mode = 1;
 
 bool encode_2d_bf16(CUtensorMap* tm, const void* base, int rows, int cols, int ld, int box_rows) {
   if (base == nullptr) return false;
@@ -368,29 +401,41 @@ bool encode_2d_bf16(CUtensorMap* tm, const void* base, int rows, int cols, int l
 
 struct Maps { CUtensorMap a, w, out, res; };
 
-template <int BN, int EPI>
+template <int BN, int EPI, int CTAS>
 cudaError_t launch_variant(const Maps& m, const TcParams& p, cudaStream_t s) {
+  using C = Cfg<BN, CTAS>;
   static bool configured = false;   // benign race: the attribute is idempotent
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(linear_tc_kernel<BN, EPI>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         Cfg<BN>::SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(linear_tc_kernel<BN, EPI, CTAS>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     configured = true;
   }
   const int total = p.tiles_m * p.tiles_n;
-  const int grid = total < g_num_sms ? total : g_num_sms;
-  linear_tc_kernel<BN, EPI><<<grid, NUM_THREADS, Cfg<BN>::SMEM_BYTES, s>>>(m.a, m.w, m.out, m.res, p);
-  return cudaGetLastError();
+  const int units = g_num_sms / CTAS;
+  const int grid = (total < units ? total : units) * CTAS;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(NUM_THREADS);
+  cfg.dynamicSmemBytes = C::SMEM_BYTES;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CTAS;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, linear_tc_kernel<BN, EPI, CTAS>, m.a, m.w, m.out, m.res, p);
 }
 
-template <int BN>
+template <int BN, int CTAS>
 cudaError_t launch_bn(int epi, const Maps& m, const TcParams& p, cudaStream_t s) {
   switch (epi) {
-    case EPI_BIAS: return launch_variant<BN, EPI_BIAS>(m, p, s);
-    case EPI_BIAS_GELU: return launch_variant<BN, EPI_BIAS_GELU>(m, p, s);
-    case EPI_BIAS_RESIDUAL: return launch_variant<BN, EPI_BIAS_RESIDUAL>(m, p, s);
-    case EPI_BIAS_POS: return launch_variant<BN, EPI_BIAS_POS>(m, p, s);
+    case EPI_BIAS: return launch_variant<BN, EPI_BIAS, CTAS>(m, p, s);
+    case EPI_BIAS_GELU: return launch_variant<BN, EPI_BIAS_GELU, CTAS>(m, p, s);
+    case EPI_BIAS_RESIDUAL: return launch_variant<BN, EPI_BIAS_RESIDUAL, CTAS>(m, p, s);
+    case EPI_BIAS_POS: return launch_variant<BN, EPI_BIAS_POS, CTAS>(m, p, s);
   }
   return cudaErrorInvalidValue;
 }
@@ -408,6 +453,7 @@ bool tc_gemm_init() {
   if (cudaGetDevice(&dev) != cudaSuccess) return false;
   if (cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
   g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  if (const char* e = getenv("VIT_GEMM_PAIR")) g_pair_mode = atoi(e);   // 0 disables the CTA-pair tiling
   return true;
 }
 
@@ -418,9 +464,13 @@ cudaError_t launch_linear_tc(const LinearArgs& a, int* dev_status, cudaStream_t 
   if ((reinterpret_cast<uintptr_t>(a.a) | reinterpret_cast<uintptr_t>(a.w) |
        reinterpret_cast<uintptr_t>(a.out) | reinterpret_cast<uintptr_t>(a.residual)) & 15)
     return cudaErrorInvalidValue;
-  const int tiles_m = (a.M + BM - 1) / BM;
-  // a full wave of 128x256 tiles, else the narrower tile to fill more SMs; shape-only decision
-  const bool wide = (long long)tiles_m * ((a.N + 255) / 256) >= g_num_sms;
+  // Shape-only choice of the tiling: CTA pairs on 256x256 tiles when they fill every pair at least
+  // once, else one CTA per 128x256 tile when that fills every SM, else 128x128 tiles.
+  const int pair_env = g_pair_mode;    // 0 = never, 1 = by shape
+  const bool pair = pair_env && a.epilogue != EPI_BIAS_POS &&
+                    (long long)((a.M + 2 * BM - 1) / (2 * BM)) * ((a.N + 255) / 256) >= g_num_sms / 2;
+  const int tiles_m = pair ? (a.M + 2 * BM - 1) / (2 * BM) : (a.M + BM - 1) / BM;
+  const bool wide = pair || (long long)tiles_m * ((a.N + 255) / 256) >= g_num_sms;
   const int bn = wide ? 256 : 128;
   TcParams p;
   p.M = a.M; p.N = a.N; p.K = a.K;
@@ -435,7 +485,7 @@ cudaError_t launch_linear_tc(const LinearArgs& a, int* dev_status, cudaStream_t 
   p.dev_status = dev_status;
   Maps m;
   if (!encode_2d_bf16(&m.a, a.a, a.M, a.K, a.lda, BM)) return cudaErrorInvalidValue;
-  if (!encode_2d_bf16(&m.w, a.w, a.N, a.K, a.ldw, bn)) return cudaErrorInvalidValue;
+  if (!encode_2d_bf16(&m.w, a.w, a.N, a.K, a.ldw, pair ? bn / 2 : bn)) return cudaErrorInvalidValue;
   // output (and residual) tiles move as 32-row x 64-column boxes through the epilogue's staging
   if (!encode_2d_bf16(&m.out, a.out, a.M, a.N, a.ldo, 32)) return cudaErrorInvalidValue;
   if (a.epilogue == EPI_BIAS_RESIDUAL) {
@@ -443,7 +493,8 @@ cudaError_t launch_linear_tc(const LinearArgs& a, int* dev_status, cudaStream_t 
   } else {
     m.res = m.out;
   }
-  return wide ? launch_bn<256>(a.epilogue, m, p, s) : launch_bn<128>(a.epilogue, m, p, s);
+  if (pair) return launch_bn<256, 2>(a.epilogue, m, p, s);
+  return wide ? launch_bn<256, 1>(a.epilogue, m, p, s) : launch_bn<128, 1>(a.epilogue, m, p, s);
 }
 
 }  // namespace vit

@@ -128,6 +128,55 @@ def oracle_images_per_s(shape, n_images, seed=0, params=None):
     return n_images / dt, cores, dt
 
 
+def microbatch_sweep(vit, model, shape, dev, torch, total=256, sizes=(1, 2, 4, 8, 16, 32, 64, 128, 256)):
+    """Microbatch sizes through an equal 4-stage partition: `total` images split into microbatches
+    issued round-robin on min(4, total/mb) streams (throughput), and one microbatch alone on one
+    stream (latency per image).  Needs max_microbatch >= the largest size that is run."""
+    counts = stage_counts(shape, 4)
+    out = []
+    pix = torch.from_numpy(vitgen.make_pixels(shape, total, seed=1)).to(dev)
+    logits = torch.empty((total, shape.num_classes), dtype=torch.float32, device=dev)
+    for mb in sizes:
+        if mb > model.cfg.max_microbatch:
+            continue
+        ns = max(1, min(4, total // mb))
+        wss, streams, wsb = model.make_pipeline_buffers(mb, ns)
+
+        def run_all():
+            model.run_pipeline(counts, mb, pix, logits, wss, streams, wsb)
+
+        def run_one():
+            model.run_pipeline(counts, mb, pix[:mb], logits[:mb], wss[:1], streams[:1], wsb)
+
+        res = {"microbatch": mb, "streams": ns}
+        for fn, key, imgs, reps in ((run_all, "images_per_s", total, 3), (run_one, "latency_ms_per_image", mb, 5)):
+            for _ in range(2):
+                fn()
+            torch.cuda.synchronize(dev)
+            t0 = time.perf_counter()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(streams[0])
+            for s in streams[1:]:
+                s.wait_event(e0)
+            for _ in range(reps):
+                fn()
+            for s in streams[1:]:
+                e = torch.cuda.Event()
+                e.record(s)
+                streams[0].wait_event(e)
+            e1.record(streams[0])
+            torch.cuda.synchronize(dev)
+            ms = e0.elapsed_time(e1) / reps
+            res[key] = imgs / (ms / 1e3) if key == "images_per_s" else ms / imgs
+            if key == "latency_ms_per_image":
+                res["latency_ms_per_microbatch"] = ms
+        for s in streams:
+            model.check(s)
+        out.append(res)
+        del wss
+    return out
+
+
 def run_reference(args, rank):
     if rank != 0:
         return
@@ -165,6 +214,8 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--workload", default="huge14", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="also run the microbatch sweep (sizes 1..256, 4 stages, streams) and add it as 'sweep'")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
 
@@ -188,12 +239,12 @@ def main():
     shape = vitgen.preset(preset)
     counts = stage_counts(shape, n_stages)
     _, blob = vitgen.make_params(shape, seed=0)
-    model = vit.VitModel(shape, blob, vit.VIT_BF16, mb, device=dev)
+    model = vit.VitModel(shape, blob, vit.VIT_BF16, max(mb, 256) if args.sweep else mb, device=dev)
     del blob
     pix_host = torch.from_numpy(vitgen.make_pixels(shape, batch, seed=rank)).pin_memory()
     pix = pix_host.to(dev)
     logits = torch.empty((batch, shape.num_classes), dtype=torch.float32, device=dev)
-    n_streams = 1
+    n_streams = max(1, min(4, batch // mb))      # microbatches round-robin on streams
     wss, streams, wsb = model.make_pipeline_buffers(mb, n_streams)
 
     def step():
@@ -228,7 +279,8 @@ def main():
 
     for _ in range(args.warmup):
         step()
-    model.check(streams[0])
+    for s_ in streams:
+        model.check(s_)
 
     launches0 = model.launches
     with ClockSampler(local) as clk:
@@ -241,7 +293,8 @@ def main():
     # per-kernel timing over the same steps (event pairs around every launch, same stream)
     vit.vit_profile_enable(model.h, True)
     prof_steps = min(args.steps, 5)
-    timed(step, prof_steps, streams)
+    # one stream for this pass, so that the event pairs of different microbatches do not overlap
+    timed(lambda: model.run_pipeline(counts, mb, pix, logits, wss[:1], streams[:1], wsb), prof_steps, streams[:1])
     prof = vit.vit_profile_collect(model.h)
     vit.vit_profile_enable(model.h, False)
 
@@ -261,6 +314,10 @@ def main():
     for s in e_streams:
         model.check(s)
     e2e_value = world * batch / (ms_e2e / 1e3)
+
+    sweep = None
+    if args.sweep:
+        sweep = microbatch_sweep(vit, model, shape, dev, torch)
 
     if rank == 0:
         pk = peaks()
@@ -292,7 +349,7 @@ def main():
             "config": {
                 "workload": f"ViT-{preset} forward, batch {batch}, microbatch {mb}, stages {counts}, "
                             f"{shape.tokens} tokens, {shape.layers} layers, hidden {shape.hidden}",
-                "global_batch": world * batch, "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                "global_batch": world * batch, "streams": n_streams, "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
                 "l2": "activations and weights per layer exceed L2 (no flush needed)",
             },
             "tflops": value * total_flops / 1e12,
@@ -317,6 +374,8 @@ def main():
             },
             "kernels": per_class,
         }
+        if sweep is not None:
+            line["sweep"] = sweep
         if not args.no_cpu_baseline and world == 1:
             n_img = 2 if preset == "huge14" else 4
             ips, cores, dt = oracle_images_per_s(shape, n_img)

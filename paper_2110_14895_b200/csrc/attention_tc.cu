@@ -158,6 +158,8 @@ attention_tc_kernel(const __grid_constant__ AttnMaps maps, const bf16* __restric
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == MMA_WARP) tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+  grid_dependency_wait();               // barrier set-up and allocation overlap the previous kernel's tail
+  grid_launch_dependents();
   // copies of the K and V rows of the keys beyond NK, as plain rows
   for (int i = threadIdx.x; i < n_extra * CH * 2; i += NUM_THREADS) {
     const int which = i / (n_extra * CH), j = i % (n_extra * CH), e = j / CH, c = j % CH;
@@ -473,8 +475,17 @@ cudaError_t launch_variant(const bf16* qkv, bf16* out, int images, int T, int he
     m.q16 = m.q64;
     m.kv16 = m.kv64;
   }
-  attention_tc_kernel<D, NK><<<images * heads, NUM_THREADS, L::BYTES, s>>>(m, qkv, out, T, heads, dev_status);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(images * heads));
+  cfg.blockDim = dim3(NUM_THREADS);
+  cfg.dynamicSmemBytes = L::BYTES;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, attention_tc_kernel<D, NK>, m, qkv, out, T, heads, dev_status);
 }
 
 }  // namespace

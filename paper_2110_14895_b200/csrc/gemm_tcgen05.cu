@@ -144,6 +144,10 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
   __syncthreads();
   if (CTAS == 2) cluster_sync();          // the peer's barriers are initialised before anyone signals them
   tc_fence_after();
+  // set-up above overlaps the tail of the previous kernel on the stream; its results are read
+  // (and its inputs overwritten) only from here on
+  grid_dependency_wait();
+  grid_launch_dependents();
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
@@ -419,13 +423,15 @@ cudaError_t launch_variant(const Maps& m, const TcParams& p, cudaStream_t s) {
   cfg.blockDim = dim3(NUM_THREADS);
   cfg.dynamicSmemBytes = C::SMEM_BYTES;
   cfg.stream = s;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = CTAS;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, linear_tc_kernel<BN, EPI, CTAS>, m.a, m.w, m.out, m.res, p);
 }
 

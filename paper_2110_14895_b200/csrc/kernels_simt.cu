@@ -32,6 +32,10 @@ layernorm_bf16_kernel(const bf16* __restrict__ x, const float* __restrict__ g,
                       int cols) {
   const int row = (int)((blockIdx.x * (size_t)blockDim.x + threadIdx.x) >> 5);
   const int lane = threadIdx.x & 31;
+  // launched with programmatic stream serialization: wait for the producer of x, then let the
+  // consumer of y start its own set-up
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (row >= rows) return;
   const int nvec = cols >> 3;
   const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)row * cols);
@@ -99,14 +103,24 @@ cudaError_t launch_layernorm_bf16(const bf16* x, const float* g, const float* b,
   const int nch = (cols / 8 + 31) / 32;
   const int threads = 256;
   const unsigned blocks = (unsigned)(((size_t)rows * 32 + threads - 1) / threads);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(blocks);
+  cfg.blockDim = dim3(threads);
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t err = cudaSuccess;
 #define LN_CASE(N) \
-  case N: layernorm_bf16_kernel<N><<<blocks, threads, 0, s>>>(x, g, b, eps, y, rows, cols); break;
+  case N: err = cudaLaunchKernelEx(&cfg, layernorm_bf16_kernel<N>, x, g, b, eps, y, rows, cols); break;
   switch (nch) {
     LN_CASE(1) LN_CASE(2) LN_CASE(3) LN_CASE(4) LN_CASE(5) LN_CASE(6) LN_CASE(7) LN_CASE(8)
     default: return cudaErrorInvalidValue;
   }
 #undef LN_CASE
-  return cudaGetLastError();
+  return err;
 }
 
 // fp32 LayerNorm: one warp per row, two passes over global memory.

@@ -177,6 +177,16 @@ __device__ __forceinline__ void cp_async_wait_all() {
 }
 
 
+// ---- programmatic dependent launch: a kernel launched with the stream-serialization attribute
+// may start while its predecessor drains; everything before grid_dependency_wait() must not
+// touch memory the predecessor reads or writes -------------------------------------------------
+__device__ __forceinline__ void grid_dependency_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+__device__ __forceinline__ void grid_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ---- CTA pairs (cta_group::2): one tcgen05.mma spans the tensor cores, shared memory and
 // tensor memory of two CTAs of a cluster; the even-ranked CTA issues it ------------------------
 __device__ __forceinline__ uint32_t cluster_ctarank() {

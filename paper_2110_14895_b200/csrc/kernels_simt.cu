@@ -39,34 +39,34 @@ layernorm_bf16_kernel(const bf16* __restrict__ x, const float* __restrict__ g,
   if (row >= rows) return;
   const int nvec = cols >> 3;
   const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)row * cols);
-  uint4 u[NCH];                       // the row stays packed (bf16) in registers between passes
+  uint4 u[NCH];
 #pragma unroll
-  for (int i = 0; i < NCH; ++i) {
+  for (int i = 0; i < NCH; ++i) {            // all loads in flight before the first use
     const int idx = lane + 32 * i;
     u[i] = idx < nvec ? __ldg(xr + idx) : make_uint4(0, 0, 0, 0);
   }
+  // bf16 -> fp32 is a shift (low half) or a mask (high half) of the 32-bit word
+  float v[NCH][8];
   float sum = 0.f;
 #pragma unroll
   for (int i = 0; i < NCH; ++i) {
-    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u[i]);
+    const uint32_t w[4] = {u[i].x, u[i].y, u[i].z, u[i].w};
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      const float2 f = __bfloat1622float2(h[e]);
-      sum += f.x + f.y;               // padded chunks are zero
+      v[i][2 * e] = __uint_as_float(w[e] << 16);
+      v[i][2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+      sum += v[i][2 * e] + v[i][2 * e + 1];          // padded chunks are zero
     }
   }
   const float mean = warp_sum(sum) / (float)cols;
   float sq = 0.f;
 #pragma unroll
   for (int i = 0; i < NCH; ++i) {
-    if (lane + 32 * i < nvec) {
-      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u[i]);
+    const bool in = lane + 32 * i < nvec;
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float2 f = __bfloat1622float2(h[e]);
-        const float c0 = f.x - mean, c1 = f.y - mean;
-        sq += c0 * c0 + c1 * c1;
-      }
+    for (int e = 0; e < 8; ++e) {
+      v[i][e] = in ? v[i][e] - mean : 0.f;
+      sq = fmaf(v[i][e], v[i][e], sq);
     }
   }
   const float rstd = 1.0f / sqrtf(warp_sum(sq) / (float)cols + eps);
@@ -81,16 +81,12 @@ layernorm_bf16_kernel(const bf16* __restrict__ x, const float* __restrict__ g,
       const float4 b1 = __ldg(reinterpret_cast<const float4*>(b) + 2 * idx + 1);
       const float gg[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
       const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u[i]);
       uint4 o;
       __nv_bfloat162* ho = reinterpret_cast<__nv_bfloat162*>(&o);
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float2 f = __bfloat1622float2(h[e]);
-        const float r0 = (f.x - mean) * rstd * gg[2 * e] + bb[2 * e];
-        const float r1 = (f.y - mean) * rstd * gg[2 * e + 1] + bb[2 * e + 1];
-        ho[e] = __floats2bfloat162_rn(r0, r1);
-      }
+      for (int e = 0; e < 4; ++e)
+        ho[e] = __floats2bfloat162_rn(v[i][2 * e] * rstd * gg[2 * e] + bb[2 * e],
+                                      v[i][2 * e + 1] * rstd * gg[2 * e + 1] + bb[2 * e + 1]);
       yr[idx] = o;
     }
   }

@@ -135,7 +135,9 @@ def _oracle_attention(qkv, images, T, heads):
 
 
 @pytest.mark.parametrize("images,T,heads,d", [(1, 5, 2, 16), (2, 197, 3, 64), (3, 257, 2, 80), (1, 32, 1, 128),
-                                              (2, 33, 2, 64), (1, 16, 1, 32), (1, 300, 1, 96)])
+                                              (2, 33, 2, 64), (1, 16, 1, 32), (1, 300, 1, 96),
+                                              (2, 258, 1, 64), (1, 260, 2, 80), (2, 193, 2, 80), (1, 208, 1, 64),
+                                              (1, 241, 1, 80), (1, 256, 2, 64)])
 @pytest.mark.parametrize("spread", [0.5, 4.0])
 def test_attention_bf16(ctx, images, T, heads, d, spread):
     vit, m = ctx

@@ -33,8 +33,30 @@ WORKLOADS = {
 }
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fc1 GEMM, from the ncu capture
 # summarised in profiles/linear_tc_kernel_huge14_shapes.md (same kernel build); None = not captured
-NCU_TRAFFIC = {"huge14": 382.1e6}
+NCU_TRAFFIC = {"huge14": 384.5e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def max_over_ranks(ms, dist=None, device=None):
+    """Slowest rank's time: the job is as fast as its slowest replica.  `dist` is torch.distributed
+    (initialised) or None for a single process."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return float(ms)
+    import torch
+    t = torch.tensor([float(ms)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_images_per_s(world, batch_per_rank, ms_per_step):
+    """Whole-job throughput of `world` independent replicas that each process `batch_per_rank`
+    images per step (weak scaling, no data-path collective)."""
+    return world * batch_per_rank / (ms_per_step / 1e3)
+
+
+def rank_pixel_seed(rank):
+    """Each replica gets its own images."""
+    return rank
 
 
 def flops_per_image(s):
@@ -241,7 +263,7 @@ def main():
     _, blob = vitgen.make_params(shape, seed=0)
     model = vit.VitModel(shape, blob, vit.VIT_BF16, max(mb, 256) if args.sweep else mb, device=dev)
     del blob
-    pix_host = torch.from_numpy(vitgen.make_pixels(shape, batch, seed=rank)).pin_memory()
+    pix_host = torch.from_numpy(vitgen.make_pixels(shape, batch, seed=rank_pixel_seed(rank))).pin_memory()
     pix = pix_host.to(dev)
     logits = torch.empty((batch, shape.num_classes), dtype=torch.float32, device=dev)
     n_streams = max(1, min(4, batch // mb))      # microbatches round-robin on streams
@@ -270,12 +292,7 @@ def main():
             stream_list[0].wait_event(e)
         ev1.record(stream_list[0])
         barrier()
-        ms = ev0.elapsed_time(ev1)
-        if world > 1:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(ev0.elapsed_time(ev1), dist if world > 1 else None, dev)
 
     for _ in range(args.warmup):
         step()
@@ -288,7 +305,7 @@ def main():
     launches = model.launches - launches0
     model.check(streams[0])
     ms_step = ms_total / args.steps
-    value = world * batch / (ms_step / 1e3)
+    value = aggregate_images_per_s(world, batch, ms_step)
 
     # per-kernel timing over the same steps (event pairs around every launch, same stream)
     vit.vit_profile_enable(model.h, True)
@@ -313,7 +330,7 @@ def main():
     ms_e2e = timed(step_host, e2e_steps, e_streams) / e2e_steps
     for s in e_streams:
         model.check(s)
-    e2e_value = world * batch / (ms_e2e / 1e3)
+    e2e_value = aggregate_images_per_s(world, batch, ms_e2e)
 
     sweep = None
     if args.sweep:

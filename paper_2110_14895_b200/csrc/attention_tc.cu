@@ -1,5 +1,5 @@
 // Fused multi-head self-attention on the 5th-generation tensor cores, for the sequence lengths
-// of ViT (T = 197 or 257 tokens; any T in [193,208] or [241,264]) and head sizes 64 and 80.
+// of ViT (T = 197 or 257 tokens; any T in [193,208] or [241,260]) and head sizes 64 and 80.
 //
 // One CTA per (image, head), two CTAs per SM.  K, V and one 128-query tile of Q are brought into
 // shared memory by TMA: columns [0,64) of the head as 128-byte-swizzled rows, columns [64,80)

@@ -41,7 +41,8 @@ enum {
   VIT_ERR_CUDA = -5,        /* a CUDA runtime/driver call or a launch failed */
   VIT_ERR_TIMEOUT = -6,     /* a bounded wait inside a kernel gave up (device status word) */
   VIT_ERR_NO_DEVICE = -7,   /* no sm_100 device / driver available */
-  VIT_ERR_TOO_LARGE = -8    /* problem exceeds the fixed scratch of an allocation-free entry point */
+  VIT_ERR_TOO_LARGE = -8,   /* problem exceeds the fixed scratch of an allocation-free entry point */
+  VIT_ERR_INFEASIBLE = -9   /* the partitioner found no assignment that fits the devices' memory */
 };
 
 enum { VIT_BF16 = 0, VIT_FP32 = 1 };
@@ -184,6 +185,38 @@ enum {
 };
 int vit_profile_enable(vit_handle* h, int on);
 int vit_profile_collect(vit_handle* h, double* ms_by_class, uint64_t* launches_by_class);
+
+/* ---- pipeline partitioner (host only, no GPU work) -------------------------------------------
+ * Chooses which consecutive layers run on which device so that the slowest pipeline stage is as
+ * fast as possible (paper Section 3.3: Eq. 1 T_comm = P_j / b(u,v); Eq. 2 T_period = max(T_comp,
+ * T_comm); Eq. 3 the transition of the three-dimensional dynamic programme over layers done,
+ * devices used and next device; Algorithm 1 with its memory check and precursor table).
+ * All pointers are host memory. */
+typedef struct vit_partition_problem {
+  int32_t layers;            /* L */
+  int32_t devices;           /* D (at most 16), or the number of categories (at most 8) */
+  const double* layer_time;  /* [D][L] seconds layer j takes on device u; T_comp of a layer range is the sum */
+  const double* out_bytes;   /* [L] P_j: bytes a stage ending with layer j sends to the next stage */
+  const double* layer_mem;   /* [L] M_j: memory layer j needs */
+  const double* device_mem;  /* [D] m_u */
+  const double* bandwidth;   /* [D][D] bytes per second from device u to device v */
+} vit_partition_problem;
+
+/* t_opt: the slowest stage's period; n_stages, stage_layers[s] (layer counts in pipeline order,
+ * summing to L) and stage_device[s] (device of stage s) describe one optimal mapping.  The two
+ * output arrays need min(L, D) entries.  Every device is used at most once; not all need be used.
+ * Errors: INVALID_ARG (null, D > 16), INFEASIBLE. */
+int vit_partition(const vit_partition_problem* problem, double* t_opt, int32_t* n_stages,
+                  int32_t* stage_layers, int32_t* stage_device);
+
+/* The same problem with identical devices grouped (paper Section 3.3, last paragraph): `devices`
+ * is the number of categories, category_count[c] the number of devices in category c, and
+ * layer_time / device_mem / bandwidth are indexed by category (bandwidth[c][c] = between two
+ * devices of category c).  stage_device receives category indices.  The state space shrinks from
+ * 2^D to prod(count + 1).  Output arrays need min(L, total devices) entries. */
+int vit_partition_categories(const vit_partition_problem* problem, const int32_t* category_count,
+                             double* t_opt, int32_t* n_stages, int32_t* stage_layers,
+                             int32_t* stage_device);
 
 /* ---- single operations, exposed so that each kernel can be checked on its own ------------
  * All pointers dev; `dtype` selects the bf16 or fp32 kernel family as in vit_config.

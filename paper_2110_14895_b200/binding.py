@@ -19,6 +19,7 @@ VIT_OK = 0
 VIT_ERR_INVALID_ARG, VIT_ERR_RANGE, VIT_ERR_CONFIG, VIT_ERR_WORKSPACE = -1, -2, -3, -4
 VIT_ERR_CUDA, VIT_ERR_TIMEOUT, VIT_ERR_NO_DEVICE = -5, -6, -7
 VIT_ERR_TOO_LARGE = -8
+VIT_ERR_INFEASIBLE = -9
 VIT_HEAD_STATIC_MAX_FLOATS = 512 * 1024
 VIT_BF16, VIT_FP32 = 0, 1
 
@@ -27,7 +28,7 @@ EXPORTS = [
     "vit_destroy", "vit_patch_embed", "vit_run_stage", "vit_head", "vit_run_pipeline",
     "vit_run_pipeline_host", "vit_check_status", "vit_launch_count", "vit_status_string",
     "vit_op_layernorm", "vit_op_linear", "vit_op_attention", "vit_profile_enable",
-    "vit_profile_collect", "vit_head_static",
+    "vit_profile_collect", "vit_head_static", "vit_partition", "vit_partition_categories",
 ]
 PROF_CLASSES = ["layernorm", "qkv", "attention", "outproj", "fc1", "fc2", "embed", "head", "op"]
 
@@ -38,6 +39,13 @@ class VitConfig(Structure):
         ("hidden", c_int32), ("layers", c_int32), ("heads", c_int32), ("mlp_dim", c_int32),
         ("num_classes", c_int32), ("ln_eps", c_float), ("dtype", c_int32),
         ("max_microbatch", c_int32),
+    ]
+
+
+class VitPartitionProblem(Structure):
+    _fields_ = [
+        ("layers", c_int32), ("devices", c_int32), ("layer_time", c_void_p), ("out_bytes", c_void_p),
+        ("layer_mem", c_void_p), ("device_mem", c_void_p), ("bandwidth", c_void_p),
     ]
 
 
@@ -93,6 +101,11 @@ def lib():
     L.vit_op_attention.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p]
     L.vit_head_static.restype = c_int
     L.vit_head_static.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p]
+    L.vit_partition.restype = c_int
+    L.vit_partition.argtypes = [P(VitPartitionProblem), P(ctypes.c_double), P(c_int32), c_void_p, c_void_p]
+    L.vit_partition_categories.restype = c_int
+    L.vit_partition_categories.argtypes = [P(VitPartitionProblem), c_void_p, P(ctypes.c_double), P(c_int32),
+                                           c_void_p, c_void_p]
     L.vit_profile_enable.restype = c_int
     L.vit_profile_enable.argtypes = [c_void_p, c_int]
     L.vit_profile_collect.restype = c_int
@@ -203,6 +216,46 @@ def vit_profile_collect(h) -> dict:
     cnt = (c_uint64 * n)()
     _check(lib().vit_profile_collect(h, ms, cnt), "vit_profile_collect")
     return {PROF_CLASSES[i]: (ms[i], int(cnt[i])) for i in range(n)}
+
+
+def _partition_call(layer_time, out_bytes, layer_mem, device_mem, bandwidth, category_count=None):
+    lt = np.ascontiguousarray(layer_time, dtype=np.float64)
+    D, Lr = lt.shape
+    ob = np.ascontiguousarray(out_bytes, dtype=np.float64)
+    lm = np.ascontiguousarray(layer_mem, dtype=np.float64)
+    dm = np.ascontiguousarray(device_mem, dtype=np.float64)
+    bw = np.ascontiguousarray(bandwidth, dtype=np.float64)
+    if ob.shape != (Lr,) or lm.shape != (Lr,) or dm.shape != (D,) or bw.shape != (D, D):
+        raise ValueError("inconsistent partition problem shapes")
+    prob = VitPartitionProblem(Lr, D, lt.ctypes.data, ob.ctypes.data, lm.ctypes.data, dm.ctypes.data, bw.ctypes.data)
+    total = D if category_count is None else int(np.sum(category_count))
+    n = max(1, min(Lr, total))
+    layers = np.zeros(n, dtype=np.int32)
+    devs = np.zeros(n, dtype=np.int32)
+    t = ctypes.c_double()
+    ns = c_int32()
+    if category_count is None:
+        st = lib().vit_partition(byref(prob), byref(t), byref(ns), layers.ctypes.data, devs.ctypes.data)
+        _check(st, "vit_partition")
+    else:
+        cc = np.ascontiguousarray(category_count, dtype=np.int32)
+        if cc.shape != (D,):
+            raise ValueError("one count per category")
+        st = lib().vit_partition_categories(byref(prob), cc.ctypes.data, byref(t), byref(ns), layers.ctypes.data,
+                                            devs.ctypes.data)
+        _check(st, "vit_partition_categories")
+    k = ns.value
+    return t.value, [(int(layers[i]), int(devs[i])) for i in range(k)]
+
+
+def vit_partition(layer_time, out_bytes, layer_mem, device_mem, bandwidth):
+    """Host-side pipeline partitioner.  Returns (T_opt, [(layer_count, device), ...])."""
+    return _partition_call(layer_time, out_bytes, layer_mem, device_mem, bandwidth)
+
+
+def vit_partition_categories(layer_time, out_bytes, layer_mem, device_mem, bandwidth, category_count):
+    """The same with identical devices grouped; devices in the result are category indices."""
+    return _partition_call(layer_time, out_bytes, layer_mem, device_mem, bandwidth, category_count)
 
 
 def vit_op_layernorm(h, dtype, rows, cols, x, gain, shift, eps, y, stream=0):

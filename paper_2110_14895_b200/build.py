@@ -8,7 +8,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(PKG, "_build")
 LIB = os.path.join(PKG, "libvit_b200.so")
-SOURCES = ["vit_capi.cu", "kernels_simt.cu", "gemm_tcgen05.cu", "attention.cu", "attention_tc.cu"]
+SOURCES = ["vit_capi.cu", "kernels_simt.cu", "gemm_tcgen05.cu", "attention.cu", "attention_tc.cu", "partition.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-Xptxas", "-v",

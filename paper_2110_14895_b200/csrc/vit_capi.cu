@@ -515,6 +515,7 @@ const char* vit_status_string(int status) {
     case VIT_ERR_CUDA: return "CUDA call or kernel launch failed";
     case VIT_ERR_TIMEOUT: return "a bounded wait inside a kernel expired";
     case VIT_ERR_NO_DEVICE: return "no usable sm_100 device";
+    case VIT_ERR_INFEASIBLE: return "no partition fits the devices' memory";
     case VIT_ERR_TOO_LARGE: return "problem larger than the fixed scratch of this allocation-free entry point";
   }
   return "unknown status";

@@ -169,6 +169,13 @@ int vit_run_pipeline_host(vit_handle* h, const int32_t* stage_layers, int n_stag
  * if the stream reported an error. */
 int vit_check_status(vit_handle* h, void* stream);
 
+/* Failure-detection self-test.  Every wait inside the tensor-core kernels is bounded: when it
+ * expires the kernel raises the device status word and returns.  This call launches a one-warp
+ * kernel whose wait can never be satisfied, with a limit of `limit_cycles` SM cycles (at most
+ * 2^31, about a second), so that the path can be exercised without a stuck kernel: afterwards
+ * vit_check_status returns VIT_ERR_TIMEOUT once and the handle keeps working. */
+int vit_debug_wait_probe(vit_handle* h, int64_t limit_cycles, void* stream);
+
 /* Number of kernels this handle has launched so far (host counter). */
 uint64_t vit_launch_count(const vit_handle* h);
 

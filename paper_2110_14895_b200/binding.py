@@ -29,6 +29,7 @@ EXPORTS = [
     "vit_run_pipeline_host", "vit_check_status", "vit_launch_count", "vit_status_string",
     "vit_op_layernorm", "vit_op_linear", "vit_op_attention", "vit_profile_enable",
     "vit_profile_collect", "vit_head_static", "vit_partition", "vit_partition_categories",
+    "vit_debug_wait_probe",
 ]
 PROF_CLASSES = ["layernorm", "qkv", "attention", "outproj", "fc1", "fc2", "embed", "head", "op"]
 
@@ -106,6 +107,8 @@ def lib():
     L.vit_partition_categories.restype = c_int
     L.vit_partition_categories.argtypes = [P(VitPartitionProblem), c_void_p, P(ctypes.c_double), P(c_int32),
                                            c_void_p, c_void_p]
+    L.vit_debug_wait_probe.restype = c_int
+    L.vit_debug_wait_probe.argtypes = [c_void_p, ctypes.c_int64, c_void_p]
     L.vit_profile_enable.restype = c_int
     L.vit_profile_enable.argtypes = [c_void_p, c_int]
     L.vit_profile_collect.restype = c_int
@@ -199,6 +202,10 @@ def vit_run_pipeline_host(h, stage_layers, batch, microbatch, host_pixels, host_
 
 def vit_check_status(h, stream=0) -> None:
     _check(lib().vit_check_status(h, stream), "vit_check_status")
+
+
+def vit_debug_wait_probe(h, limit_cycles, stream=0) -> None:
+    _check(lib().vit_debug_wait_probe(h, int(limit_cycles), stream), "vit_debug_wait_probe")
 
 
 def vit_launch_count(h) -> int:

@@ -448,6 +448,27 @@ cudaError_t launch_bn(int epi, const Maps& m, const TcParams& p, cudaStream_t s)
 
 }  // namespace
 
+// A wait that nothing ever satisfies, with a short limit: shows the path a stuck kernel takes
+// (status word raised, kernel returns, context stays usable) without hanging anything.
+namespace {
+__global__ void wait_probe_kernel(long long limit_cycles, int* dev_status) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    ptx::mbar_init(ptx::smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (!ptx::mbar_wait_limit(ptx::smem_u32(&bar), 0, &abort_flag, limit_cycles))
+      atomicExch(dev_status, (int)VIT_ERR_TIMEOUT);
+  }
+}
+}  // namespace
+
+cudaError_t launch_wait_probe(long long limit_cycles, int* dev_status, cudaStream_t s) {
+  wait_probe_kernel<<<1, 32, 0, s>>>(limit_cycles, dev_status);
+  return cudaGetLastError();
+}
+
 bool tc_gemm_init() {
   if (g_encode) return true;
   void* fn = nullptr;

@@ -503,6 +503,13 @@ int vit_profile_collect(vit_handle* h, double* ms_by_class, uint64_t* launches_b
   return st;
 }
 
+int vit_debug_wait_probe(vit_handle* h, int64_t limit_cycles, void* stream) {
+  if (!h || limit_cycles < 1 || limit_cycles > (1ll << 31)) return VIT_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  VIT_LAUNCH(h, VIT_PROF_OP, launch_wait_probe(limit_cycles, h->dev_status, s));
+  return VIT_OK;
+}
+
 uint64_t vit_launch_count(const vit_handle* h) { return h ? h->launches.load() : 0; }
 
 const char* vit_status_string(int status) {

@@ -92,6 +92,8 @@ cudaError_t launch_head_static(const void* tokens, const float* g, const float* 
                                const void* W, const float* bias, float* logits, int images, int T,
                                int H, int classes, bool act_bf16, cudaStream_t s);
 
+cudaError_t launch_wait_probe(long long limit_cycles, int* dev_status, cudaStream_t s);
+
 bool tc_gemm_init();   // resolves the driver's tensor-map encoder; false if unavailable
 
 }  // namespace vit

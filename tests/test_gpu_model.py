@@ -218,3 +218,22 @@ def test_huge14_microbatch_sweep_on_streams_is_consistent():
             assert ok, (mb, msg)
         del wss
     m.close()
+
+
+def test_bounded_wait_raises_status_and_leaves_the_handle_usable():
+    """A wait nothing satisfies expires after its (short) limit: the status word reports it once,
+    nothing hangs, and the same handle then runs a stage correctly."""
+    shape = vitgen.preset("tiny16").with_(layers=2)
+    vit, m, _ = _model(shape, _vit().VIT_BF16, 1)
+    x = torch.randn((1, m.T, shape.hidden), device="cuda").to(torch.bfloat16)
+    ref = m.run_stage(0, 2, x)
+    m.check()
+    vit.vit_debug_wait_probe(m.h, 2_000_000)          # about a millisecond
+    with pytest.raises(vit.VitError) as e:
+        m.check()
+    assert e.value.status == vit.VIT_ERR_TIMEOUT
+    m.check()                                          # the word was cleared by the read
+    again = m.run_stage(0, 2, x)
+    m.check()
+    assert torch.equal(ref, again)
+    m.close()

@@ -491,13 +491,20 @@ cudaError_t launch_linear_tc(const LinearArgs& a, int* dev_status, cudaStream_t 
   if ((reinterpret_cast<uintptr_t>(a.a) | reinterpret_cast<uintptr_t>(a.w) |
        reinterpret_cast<uintptr_t>(a.out) | reinterpret_cast<uintptr_t>(a.residual)) & 15)
     return cudaErrorInvalidValue;
-  // Shape-only choice of the tiling: CTA pairs on 256x256 tiles when they fill every pair at least
-  // once, else one CTA per 128x256 tile when that fills every SM, else 128x128 tiles.
-  const int pair_env = g_pair_mode;    // 0 = never, 1 = by shape
-  const bool pair = pair_env && a.epilogue != EPI_BIAS_POS &&
-                    (long long)((a.M + 2 * BM - 1) / (2 * BM)) * ((a.N + 255) / 256) >= g_num_sms / 2;
-  const int tiles_m = pair ? (a.M + 2 * BM - 1) / (2 * BM) : (a.M + BM - 1) / BM;
-  const bool wide = pair || (long long)tiles_m * ((a.N + 255) / 256) >= g_num_sms;
+  // Shape-only choice of the tiling by a small cost model: rounds of the static schedule times
+  // the per-SM work of one tile (128x256 = 1 for a pair or a single CTA, 128x128 = 0.5, measured nearer 0.75), with a
+  // bonus for the pair tiling's lower load traffic and a penalty for the small tile's overheads.
+  const long long nt256 = (a.N + 255) / 256, nt128 = (a.N + 127) / 128;
+  const long long tm1 = (a.M + BM - 1) / BM, tm2 = (a.M + 2 * BM - 1) / (2 * BM);
+  const long long units1 = g_num_sms, units2 = g_num_sms / 2;
+  auto rounds = [](long long tiles, long long units) { return (double)((tiles + units - 1) / units); };
+  const double cost_pair = (g_pair_mode && a.epilogue != EPI_BIAS_POS && units2 > 0)
+                               ? 0.92 * rounds(tm2 * nt256, units2) : 1e30;
+  const double cost_256 = 1.0 * rounds(tm1 * nt256, units1);
+  const double cost_128 = 0.75 * rounds(tm1 * nt128, units1);
+  const bool pair = cost_pair <= cost_256 && cost_pair <= cost_128;
+  const bool wide = pair || cost_256 <= cost_128;
+  const int tiles_m = (int)(pair ? tm2 : tm1);
   const int bn = wide ? 256 : 128;
   TcParams p;
   p.M = a.M; p.N = a.N; p.K = a.K;

@@ -199,6 +199,16 @@ def microbatch_sweep(vit, model, shape, dev, torch, total=256, sizes=(1, 2, 4, 8
     return out
 
 
+def workload_config(preset, shape, batch, mb, counts, world, n_streams):
+    return {
+        "workload": f"ViT-{preset} forward, batch {batch}, microbatch {mb}, stages {counts}, "
+                    f"{shape.tokens} tokens, {shape.layers} layers, hidden {shape.hidden}",
+        "global_batch": world * batch, "streams": n_streams,
+        "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+        "l2": "activations and weights per layer exceed L2 (no flush needed)",
+    }
+
+
 def run_reference(args, rank):
     if rank != 0:
         return
@@ -218,8 +228,8 @@ def run_reference(args, rank):
         "impl": "reference", "metric": "images/sec", "value": value, "unit": "images/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"ViT-{preset} forward, {shape.tokens} tokens, {shape.layers} layers",
-                   "images_per_step": per_step},
+        "config": workload_config(preset, shape, batch, mb, stage_counts(shape, n_stages), 1,
+                                  max(1, min(4, batch // mb))) | {"reference_images_per_step": per_step},
         "cpu_baseline": {"value": value, "unit": "images/s", "cores": cores, "kind": "oracle",
                          "sample": f"{per_step} image per step of the {preset} workload, numpy fp64"},
         "e2e": {"value": value, "unit": "images/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -363,12 +373,7 @@ def main():
             "metric": "images/sec", "value": value, "unit": "images/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {
-                "workload": f"ViT-{preset} forward, batch {batch}, microbatch {mb}, stages {counts}, "
-                            f"{shape.tokens} tokens, {shape.layers} layers, hidden {shape.hidden}",
-                "global_batch": world * batch, "streams": n_streams, "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
-                "l2": "activations and weights per layer exceed L2 (no flush needed)",
-            },
+            "config": workload_config(preset, shape, batch, mb, counts, world, n_streams),
             "tflops": value * total_flops / 1e12,
             "frac_of_bf16_peak": {"burst": value * total_flops / 1e12 / world / pk["bf16_tflops"],
                                   "sustained": value * total_flops / 1e12 / world / pk["bf16_tflops_sustained"],

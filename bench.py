@@ -32,7 +32,7 @@ WORKLOADS = {
     "base16": ("base16", 64, 16, 4),
 }
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fc1 GEMM, from the ncu capture
-# summarised in profiles/linear_tc_kernel_huge14_shapes.md (same kernel build); None = not captured
+# whose summary is kept under profiles/ (same kernel build); None = not captured
 NCU_TRAFFIC = {"huge14": 384.5e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 

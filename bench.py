@@ -30,6 +30,7 @@ WORKLOADS = {
     "huge14": ("huge14", 128, 128, 1),
     "large16": ("large16", 128, 8, 16),
     "base16": ("base16", 64, 16, 4),
+    "small16": ("small16", 64, 16, 4),
 }
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fc1 GEMM, from the ncu capture
 # whose summary is kept under profiles/ (same kernel build); None = not captured

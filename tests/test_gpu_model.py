@@ -151,6 +151,11 @@ def test_base16_batch64_four_microbatches_four_stages():
     m.close()
 
 
+def test_small16_batch32_two_microbatches_three_stages():
+    _, m, _, _ = _pipeline_vs_oracle("small16", 32, 16, [(0, 5), (5, 6), (6, 12)], 2, [0, 15, 16, 31])
+    m.close()
+
+
 def test_base16_host_buffers_pipeline():
     _, m, _, _ = _pipeline_vs_oracle("base16", 8, 4, vitgen.equal_partition(4, 12), 2, [0, 3, 4, 7], host=True)
     m.close()

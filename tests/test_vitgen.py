@@ -27,6 +27,7 @@ def test_param_counts():
     assert vitgen.param_count(vitgen.preset("base16")) == 86_567_656
     assert vitgen.param_count(vitgen.preset("large16")) == 304_326_632
     assert vitgen.param_count(vitgen.preset("huge14")) == 632_045_800
+    assert vitgen.param_count(vitgen.preset("small16")) == 22_050_664
 
 
 def test_blob_views_and_pack_roundtrip():

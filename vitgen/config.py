@@ -43,6 +43,8 @@ PRESETS = {
     "base16": ViTConfig(patch_size=16, hidden=768, layers=12, heads=12, mlp_dim=3072),
     "large16": ViTConfig(patch_size=16, hidden=1024, layers=24, heads=16, mlp_dim=4096),
     "huge14": ViTConfig(patch_size=14, hidden=1280, layers=32, heads=16, mlp_dim=5120),
+    # the shape of the "small" compressed model family (same structure, smaller dimensions)
+    "small16": ViTConfig(patch_size=16, hidden=384, layers=12, heads=6, mlp_dim=1536),
 }
 
 

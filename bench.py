@@ -247,6 +247,7 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--workload", default="huge14", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--streams", type=int, default=0, help="streams for the stage runner (0 = min(4, microbatches))")
     ap.add_argument("--sweep", action="store_true",
                     help="also run the microbatch sweep (sizes 1..256, 4 stages, streams) and add it as 'sweep'")
     args = ap.parse_args()
@@ -277,7 +278,7 @@ def main():
     pix_host = torch.from_numpy(vitgen.make_pixels(shape, batch, seed=rank_pixel_seed(rank))).pin_memory()
     pix = pix_host.to(dev)
     logits = torch.empty((batch, shape.num_classes), dtype=torch.float32, device=dev)
-    n_streams = max(1, min(4, batch // mb))      # microbatches round-robin on streams
+    n_streams = args.streams if args.streams > 0 else max(1, min(4, batch // mb))   # microbatches round-robin on streams
     wss, streams, wsb = model.make_pipeline_buffers(mb, n_streams)
 
     def step():

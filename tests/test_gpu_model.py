@@ -242,3 +242,36 @@ def test_bounded_wait_raises_status_and_leaves_the_handle_usable():
     m.check()
     assert torch.equal(ref, again)
     m.close()
+
+
+def test_pipeline_ragged_last_microbatch_and_argument_errors():
+    """Batch 5 in microbatches of 2 leaves a last microbatch of one image; stage counts must sum
+    to the layer count; a failed call launches nothing."""
+    shape = vitgen.preset("tiny16").with_(layers=4)
+    vit, m, params = _model(shape, _vit().VIT_BF16, 2)
+    pix = vitgen.make_pixels(shape, 5, seed=2)
+    dp = torch.from_numpy(pix).cuda()
+    wss, streams, wsb = m.make_pipeline_buffers(2, 2)
+    logits = torch.full((5, shape.num_classes), float("nan"), dtype=torch.float32, device="cuda")
+    torch.cuda.synchronize()
+    m.run_pipeline([1, 3], 2, dp, logits, wss, streams, wsb)
+    for s in streams:
+        m.check(s)
+    want = O.forward(params, shape, pix)
+    ok, msg = logits_within_tolerance(logits.cpu().numpy(), want, 2e-2, 0.9995)
+    assert ok, msg
+    one = m.forward(dp[4:5])                      # the ragged microbatch equals a batch-of-one call
+    assert torch.equal(one, logits[4:5])
+    before = m.launches
+    for counts, status in (([1, 2], vit.VIT_ERR_RANGE), ([4, 0], vit.VIT_ERR_RANGE), ([], vit.VIT_ERR_INVALID_ARG)):
+        with pytest.raises(vit.VitError) as e:
+            m.run_pipeline(counts, 2, dp, logits, wss, streams, wsb)
+        assert e.value.status == status
+    with pytest.raises(vit.VitError) as e:
+        m.run_pipeline([4], 3, dp, logits, wss, streams, wsb)      # microbatch above max_microbatch
+    assert e.value.status == vit.VIT_ERR_INVALID_ARG
+    with pytest.raises(vit.VitError) as e:
+        m.run_pipeline([4], 2, dp, logits, wss, streams, 1024)     # workspace too small
+    assert e.value.status == vit.VIT_ERR_WORKSPACE
+    assert m.launches == before
+    m.close()

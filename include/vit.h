@@ -41,7 +41,8 @@ enum {
   VIT_ERR_CUDA = -5,        /* a CUDA runtime/driver call or a launch failed */
   VIT_ERR_TIMEOUT = -6,     /* a bounded wait inside a kernel gave up (device status word) */
   VIT_ERR_NO_DEVICE = -7,   /* no sm_100 device / driver available */
-  VIT_ERR_TOO_LARGE = -8,   /* problem exceeds the fixed scratch of an allocation-free entry point */
+  VIT_ERR_TOO_LARGE = -8,   /* problem exceeds the fixed scratch of an allocation-free entry point,
+                               or the partitioner's tables do not fit in host memory */
   VIT_ERR_INFEASIBLE = -9   /* the partitioner found no assignment that fits the devices' memory */
 };
 
@@ -212,7 +213,9 @@ typedef struct vit_partition_problem {
 /* t_opt: the slowest stage's period; n_stages, stage_layers[s] (layer counts in pipeline order,
  * summing to L) and stage_device[s] (device of stage s) describe one optimal mapping.  The two
  * output arrays need min(L, D) entries.  Every device is used at most once; not all need be used.
- * Errors: INVALID_ARG (null, D > 16), INFEASIBLE. */
+ * Errors: INVALID_ARG (null pointer, D > 16, a bandwidth that is not positive, a time, size or
+ * memory that is negative or not a number), INFEASIBLE, TOO_LARGE (the tables of the dynamic
+ * programme, about 8 * L * 2^D * D bytes, could not be allocated). */
 int vit_partition(const vit_partition_problem* problem, double* t_opt, int32_t* n_stages,
                   int32_t* stage_layers, int32_t* stage_device);
 

@@ -13,8 +13,11 @@
  *     PyTorch tensor) and must stay alive until the stream has drained.  They must be 16-byte
  *     aligned.  "host" pointers are ordinary (preferably pinned) host memory.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls are
- *     asynchronous on that stream, allocate nothing and never synchronise the host, except
- *     where stated.
+ *     asynchronous on that stream, allocate no device memory and never synchronise the host,
+ *     except where stated (while vit_profile_enable is on, every launch also creates a pair of
+ *     CUDA events).
+ *   - A handle belongs to the CUDA device that was current in vit_create; every call that takes
+ *     the handle must be made with that device current (otherwise VIT_ERR_INVALID_ARG).
  *   - Activations are row-major [microbatch, T, H] (T = patches + 1 class token, H = hidden).
  *     Their element type is the model's activation type: bf16 when config.dtype == VIT_BF16
  *     (bf16 operands, fp32 accumulation), fp32 when config.dtype == VIT_FP32.
@@ -165,9 +168,12 @@ int vit_run_pipeline_host(vit_handle* h, const int32_t* stage_layers, int n_stag
                           void* const* ws_per_stream, size_t ws_bytes, void* const* streams,
                           int n_streams);
 
-/* Synchronises `stream`, then returns and clears the device status word: VIT_OK, or
- * VIT_ERR_TIMEOUT if a bounded wait in a kernel gave up since the last check, or VIT_ERR_CUDA
- * if the stream reported an error. */
+/* Returns and clears the device status word after everything queued on `stream` has finished
+ * (synchronises that stream): VIT_OK, or VIT_ERR_TIMEOUT if a bounded wait in a kernel gave up
+ * since the last check, or VIT_ERR_CUDA if the stream reported an error.  There is one word per
+ * handle, shared by all its streams; it is read and cleared in one atomic step on the device, so
+ * a timeout raised on another stream while this call runs is reported by the next check.  To
+ * know that a multi-stream run was clean, check after each of its streams. */
 int vit_check_status(vit_handle* h, void* stream);
 
 /* Failure-detection self-test.  Every wait inside the tensor-core kernels is bounded: when it
@@ -242,6 +248,14 @@ int vit_op_layernorm(vit_handle* h, int dtype, int rows, int cols, const void* x
  * bf16 family: K % 8 == 0 and N % 8 == 0. */
 int vit_op_linear(vit_handle* h, int dtype, int M, int N, int K, const void* a, const void* w,
                   const float* bias, int epilogue, const void* residual, void* out, void* stream);
+
+/* vit_op_linear with the tiling of the bf16 tensor-core kernel chosen by the caller instead of
+ * by the library's shape-only cost model, so that every tiling can be checked on any shape.
+ * VIT_TILING_PAIR_256x256 runs CTA pairs on 256 x 256 tiles.  fp32 family: AUTO only. */
+enum { VIT_TILING_AUTO = 0, VIT_TILING_128x128 = 1, VIT_TILING_128x256 = 2, VIT_TILING_PAIR_256x256 = 3 };
+int vit_op_linear_tiled(vit_handle* h, int dtype, int M, int N, int K, const void* a, const void* w,
+                        const float* bias, int epilogue, const void* residual, void* out, int tiling,
+                        void* stream);
 
 /* Multi-head self-attention for `images` sequences of T tokens: qkv [images*T, 3*heads*d]
  * (column blocks Q, K, V; head-major inside each), out [images*T, heads*d];

@@ -22,12 +22,13 @@ VIT_ERR_TOO_LARGE = -8
 VIT_ERR_INFEASIBLE = -9
 VIT_HEAD_STATIC_MAX_FLOATS = 512 * 1024
 VIT_BF16, VIT_FP32 = 0, 1
+VIT_TILING_AUTO, VIT_TILING_128x128, VIT_TILING_128x256, VIT_TILING_PAIR_256x256 = 0, 1, 2, 3
 
 EXPORTS = [
     "vit_param_count", "vit_workspace_bytes", "vit_pipeline_workspace_bytes", "vit_create",
     "vit_destroy", "vit_patch_embed", "vit_run_stage", "vit_head", "vit_run_pipeline",
     "vit_run_pipeline_host", "vit_check_status", "vit_launch_count", "vit_status_string",
-    "vit_op_layernorm", "vit_op_linear", "vit_op_attention", "vit_profile_enable",
+    "vit_op_layernorm", "vit_op_linear", "vit_op_linear_tiled", "vit_op_attention", "vit_profile_enable",
     "vit_profile_collect", "vit_head_static", "vit_partition", "vit_partition_categories",
     "vit_debug_wait_probe",
 ]
@@ -98,6 +99,8 @@ def lib():
     L.vit_op_layernorm.argtypes = [c_void_p, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_float, c_void_p, c_void_p]
     L.vit_op_linear.restype = c_int
     L.vit_op_linear.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p]
+    L.vit_op_linear_tiled.restype = c_int
+    L.vit_op_linear_tiled.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_int, c_void_p]
     L.vit_op_attention.restype = c_int
     L.vit_op_attention.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p]
     L.vit_head_static.restype = c_int
@@ -271,6 +274,11 @@ def vit_op_layernorm(h, dtype, rows, cols, x, gain, shift, eps, y, stream=0):
 
 def vit_op_linear(h, dtype, M, N, K, a, w, bias, epilogue, residual, out, stream=0):
     _check(lib().vit_op_linear(h, dtype, M, N, K, a, w, bias, epilogue, residual, out, stream), "vit_op_linear")
+
+
+def vit_op_linear_tiled(h, dtype, M, N, K, a, w, bias, epilogue, residual, out, tiling, stream=0):
+    _check(lib().vit_op_linear_tiled(h, dtype, M, N, K, a, w, bias, epilogue, residual, out, tiling, stream),
+           "vit_op_linear_tiled")
 
 
 def vit_op_attention(h, dtype, images, T, heads, d, qkv, out, stream=0):

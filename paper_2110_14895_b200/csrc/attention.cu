@@ -176,13 +176,9 @@ attention_bf16_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ out, int 
 template <int D, int NT, int MINB>
 cudaError_t launch_variant(const bf16* qkv, bf16* out, int images, int T, int heads, int nw, size_t smem,
                            cudaStream_t s) {
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(attention_bf16_kernel<D, NT, MINB>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static PerDeviceFlag configured;
+  cudaError_t e = ensure_dynamic_smem(configured, attention_bf16_kernel<D, NT, MINB>, 227 * 1024);
+  if (e != cudaSuccess) return e;
   attention_bf16_kernel<D, NT, MINB><<<images * heads, nw * 32, smem, s>>>(qkv, out, T, heads);
   return cudaGetLastError();
 }
@@ -214,6 +210,7 @@ cudaError_t launch_attention_bf16(const bf16* qkv, bf16* out, int images, int T,
     case 64: return launch_d<64>(qkv, out, images, T, heads, s);
     case 80: return launch_d<80>(qkv, out, images, T, heads, s);
     case 96: return launch_d<96>(qkv, out, images, T, heads, s);
+    case 112: return launch_d<112>(qkv, out, images, T, heads, s);
     case 128: return launch_d<128>(qkv, out, images, T, heads, s);
   }
   return cudaErrorInvalidValue;

@@ -457,13 +457,9 @@ cudaError_t launch_variant(const bf16* qkv, bf16* out, int images, int T, int he
       return cudaErrorNotReady;
     g_encode = reinterpret_cast<EncodeTiledFn>(fn);
   }
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel<D, NK>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::BYTES);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static PerDeviceFlag configured;
+  cudaError_t e = ensure_dynamic_smem(configured, attention_tc_kernel<D, NK>, (int)L::BYTES);
+  if (e != cudaSuccess) return e;
   const size_t rows = (size_t)images * T, cols = (size_t)3 * heads * D;
   AttnMaps m;
   if (!encode_map(&m.q64, qkv, rows, cols, 64, QT, CU_TENSOR_MAP_SWIZZLE_128B)) return cudaErrorInvalidValue;

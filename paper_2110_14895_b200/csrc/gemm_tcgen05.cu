@@ -18,7 +18,6 @@
 #include "sm100_ptx.cuh"
 
 #include <cuda.h>
-#include <cstdlib>
 
 namespace vit {
 
@@ -389,8 +388,6 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
-int g_num_sms = 0;
-int g_pair_mode = 1;
 
 bool encode_2d_bf16(CUtensorMap* tm, const void* base, int rows, int cols, int ld, int box_rows) {
   if (base == nullptr) return false;
@@ -408,15 +405,11 @@ struct Maps { CUtensorMap a, w, out, res; };
 template <int BN, int EPI, int CTAS>
 cudaError_t launch_variant(const Maps& m, const TcParams& p, cudaStream_t s) {
   using C = Cfg<BN, CTAS>;
-  static bool configured = false;   // benign race: the attribute is idempotent
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(linear_tc_kernel<BN, EPI, CTAS>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static PerDeviceFlag configured;
+  cudaError_t e = ensure_dynamic_smem(configured, linear_tc_kernel<BN, EPI, CTAS>, C::SMEM_BYTES);
+  if (e != cudaSuccess) return e;
   const int total = p.tiles_m * p.tiles_n;
-  const int units = g_num_sms / CTAS;
+  const int units = current_device_sm_count() / CTAS;
   const int grid = (total < units ? total : units) * CTAS;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
@@ -464,6 +457,15 @@ __global__ void wait_probe_kernel(long long limit_cycles, int* dev_status) {
 }
 }  // namespace
 
+namespace {
+__global__ void status_take_kernel(int* status, int* snapshot) { *snapshot = atomicExch(status, 0); }
+}  // namespace
+
+cudaError_t launch_status_take(int* status, int* snapshot, cudaStream_t s) {
+  status_take_kernel<<<1, 1, 0, s>>>(status, snapshot);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_wait_probe(long long limit_cycles, int* dev_status, cudaStream_t s) {
   wait_probe_kernel<<<1, 32, 0, s>>>(limit_cycles, dev_status);
   return cudaGetLastError();
@@ -476,12 +478,20 @@ bool tc_gemm_init() {
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
       q != cudaDriverEntryPointSuccess || fn == nullptr)
     return false;
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return false;
-  if (cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
   g_encode = reinterpret_cast<EncodeTiledFn>(fn);
-  if (const char* e = getenv("VIT_GEMM_PAIR")) g_pair_mode = atoi(e);   // 0 disables the CTA-pair tiling
-  return true;
+  return current_device_sm_count() > 0;
+}
+
+int current_device_sm_count() {
+  static std::atomic<int> cache[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  const bool tracked = dev >= 0 && dev < 64;
+  int n = tracked ? cache[dev].load(std::memory_order_relaxed) : 0;
+  if (n > 0) return n;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+  if (tracked) cache[dev].store(n, std::memory_order_relaxed);
+  return n;
 }
 
 cudaError_t launch_linear_tc(const LinearArgs& a, int* dev_status, cudaStream_t s) {
@@ -496,14 +506,25 @@ cudaError_t launch_linear_tc(const LinearArgs& a, int* dev_status, cudaStream_t 
   // bonus for the pair tiling's lower load traffic and a penalty for the small tile's overheads.
   const long long nt256 = (a.N + 255) / 256, nt128 = (a.N + 127) / 128;
   const long long tm1 = (a.M + BM - 1) / BM, tm2 = (a.M + 2 * BM - 1) / (2 * BM);
-  const long long units1 = g_num_sms, units2 = g_num_sms / 2;
+  const int sms = current_device_sm_count();
+  if (sms < 2) return cudaErrorInvalidDevice;
+  const long long units1 = sms, units2 = sms / 2;
   auto rounds = [](long long tiles, long long units) { return (double)((tiles + units - 1) / units); };
-  const double cost_pair = (g_pair_mode && a.epilogue != EPI_BIAS_POS && units2 > 0)
-                               ? 0.92 * rounds(tm2 * nt256, units2) : 1e30;
+  const bool pair_allowed = a.epilogue != EPI_BIAS_POS;    // the scatter epilogue has no pair variant
+  const double cost_pair = pair_allowed ? 0.92 * rounds(tm2 * nt256, units2) : 1e30;
   const double cost_256 = 1.0 * rounds(tm1 * nt256, units1);
   const double cost_128 = 0.75 * rounds(tm1 * nt128, units1);
-  const bool pair = cost_pair <= cost_256 && cost_pair <= cost_128;
-  const bool wide = pair || cost_256 <= cost_128;
+  bool pair = cost_pair <= cost_256 && cost_pair <= cost_128;
+  bool wide = pair || cost_256 <= cost_128;
+  switch (a.tiling) {
+    case TILING_AUTO: break;
+    case TILING_128x128: pair = false; wide = false; break;
+    case TILING_128x256: pair = false; wide = true; break;
+    case TILING_PAIR_256x256:
+      if (!pair_allowed) return cudaErrorInvalidValue;
+      pair = true; wide = true; break;
+    default: return cudaErrorInvalidValue;
+  }
   const int tiles_m = (int)(pair ? tm2 : tm1);
   const int bn = wide ? 256 : 128;
   TcParams p;

@@ -6,6 +6,7 @@
 #include <cuda_bf16.h>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <thread>
 #include <vector>
@@ -143,8 +144,15 @@ int linear(Handle* h, int cls, const LinearArgs& a, cudaStream_t s) {
   return VIT_OK;
 }
 
+// A handle's parameters, status word and kernel attributes live on the device it was created on.
+bool on_own_device(const vit_handle* h) {
+  int dev = -1;
+  return h && cudaGetDevice(&dev) == cudaSuccess && dev == h->device;
+}
+
 int check_call(const vit_handle* h, int mb, const void* ws, size_t ws_bytes, size_t need) {
   if (!h || mb < 1 || mb > h->cfg.max_microbatch || !ws || misaligned(ws)) return VIT_ERR_INVALID_ARG;
+  if (!on_own_device(h)) return VIT_ERR_INVALID_ARG;
   if (ws_bytes < need) return VIT_ERR_WORKSPACE;
   return VIT_OK;
 }
@@ -163,7 +171,7 @@ int run_pipeline(vit_handle* h, const int32_t* stage_layers, int n_stages, int b
                  const float* pixels, float* logits, void* const* wss, size_t ws_bytes,
                  void* const* streams, int n_streams, bool host_io) {
   if (!h || !pixels || !logits || !wss || !streams || n_streams < 1 || batch < 1 || mb < 1 ||
-      mb > h->cfg.max_microbatch)
+      mb > h->cfg.max_microbatch || !on_own_device(h))
     return VIT_ERR_INVALID_ARG;
   if (!host_io && (misaligned(pixels) || misaligned(logits))) return VIT_ERR_INVALID_ARG;
   int st = check_stages(h, stage_layers, n_stages);
@@ -302,15 +310,16 @@ int vit_create(const vit_config* cfg, const float* host_params, size_t n_params,
   void* dev_blob = nullptr;
   int* dev_status = nullptr;
   if (cudaMalloc(&dev_blob, blob_bytes) != cudaSuccess) { free(staging); return VIT_ERR_CUDA; }
-  if (cudaMalloc(&dev_status, sizeof(int)) != cudaSuccess) { cudaFree(dev_blob); free(staging); return VIT_ERR_CUDA; }
+  if (cudaMalloc(&dev_status, 2 * sizeof(int)) != cudaSuccess) { cudaFree(dev_blob); free(staging); return VIT_ERR_CUDA; }
   cudaError_t e = cudaMemcpy(dev_blob, staging, blob_bytes, cudaMemcpyHostToDevice);
   free(staging);
-  if (e == cudaSuccess) e = cudaMemset(dev_status, 0, sizeof(int));
+  if (e == cudaSuccess) e = cudaMemset(dev_status, 0, 2 * sizeof(int));
   if (e != cudaSuccess) { cudaFree(dev_blob); cudaFree(dev_status); return VIT_ERR_CUDA; }
 
   vit_handle* h = new (std::nothrow) vit_handle();
   if (!h) { cudaFree(dev_blob); cudaFree(dev_status); return VIT_ERR_CUDA; }
   h->cfg = *cfg;
+  h->device = dev;
   h->T = s.T; h->n_patches = s.Np; h->d = s.d; h->patch_k = s.Kpe; h->patch_k_pad = s.Kpad;
   h->act_bytes = act;
   h->dev_blob = dev_blob;
@@ -444,7 +453,7 @@ int vit_head(vit_handle* h, int mb, const void* tokens, float* logits, void* ws,
 }
 
 int vit_head_static(vit_handle* h, int mb, const void* tokens, float* logits, void* stream) {
-  if (!h || mb < 1 || mb > h->cfg.max_microbatch) return VIT_ERR_INVALID_ARG;
+  if (!h || mb < 1 || mb > h->cfg.max_microbatch || !on_own_device(h)) return VIT_ERR_INVALID_ARG;
   if (!tokens || !logits || misaligned(tokens) || misaligned(logits)) return VIT_ERR_INVALID_ARG;
   const vit_config& c = h->cfg;
   if ((size_t)mb * (size_t)c.hidden > (size_t)VIT_HEAD_STATIC_MAX_FLOATS) return VIT_ERR_TOO_LARGE;
@@ -471,11 +480,15 @@ int vit_run_pipeline_host(vit_handle* h, const int32_t* stage_layers, int n_stag
 }
 
 int vit_check_status(vit_handle* h, void* stream) {
-  if (!h) return VIT_ERR_INVALID_ARG;
-  if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return VIT_ERR_CUDA;
+  if (!h || !on_own_device(h)) return VIT_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // The word is read and cleared in one atomic step on the device, so a timeout raised by a
+  // kernel on another stream in the meantime is kept for the next check instead of being lost.
+  std::lock_guard<std::mutex> lock(h->status_mutex);    // one snapshot slot per handle
+  if (launch_status_take(h->dev_status, h->dev_status + 1, s) != cudaSuccess) return VIT_ERR_CUDA;
   int v = 0;
-  if (cudaMemcpy(&v, h->dev_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return VIT_ERR_CUDA;
-  if (v != 0) cudaMemset(h->dev_status, 0, sizeof(int));
+  if (cudaMemcpyAsync(&v, h->dev_status + 1, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return VIT_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return VIT_ERR_CUDA;
   return v;
 }
 
@@ -504,7 +517,7 @@ int vit_profile_collect(vit_handle* h, double* ms_by_class, uint64_t* launches_b
 }
 
 int vit_debug_wait_probe(vit_handle* h, int64_t limit_cycles, void* stream) {
-  if (!h || limit_cycles < 1 || limit_cycles > (1ll << 31)) return VIT_ERR_INVALID_ARG;
+  if (!h || limit_cycles < 1 || limit_cycles > (1ll << 31) || !on_own_device(h)) return VIT_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   VIT_LAUNCH(h, VIT_PROF_OP, launch_wait_probe(limit_cycles, h->dev_status, s));
   return VIT_OK;
@@ -530,7 +543,7 @@ const char* vit_status_string(int status) {
 
 int vit_op_layernorm(vit_handle* h, int dtype, int rows, int cols, const void* x, const float* gain,
                      const float* shift, float eps, void* y, void* stream) {
-  if (!h || !x || !gain || !shift || !y || rows < 0 || cols < 1) return VIT_ERR_INVALID_ARG;
+  if (!h || !x || !gain || !shift || !y || rows < 0 || cols < 1 || !on_own_device(h)) return VIT_ERR_INVALID_ARG;
   if (misaligned(x) || misaligned(y) || misaligned(gain) || misaligned(shift)) return VIT_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (dtype == VIT_BF16) VIT_LAUNCH(h, VIT_PROF_LAYERNORM, launch_layernorm_bf16((const bf16*)x, gain, shift, eps, (bf16*)y, rows, cols, s));
@@ -541,13 +554,22 @@ int vit_op_layernorm(vit_handle* h, int dtype, int rows, int cols, const void* x
 
 int vit_op_linear(vit_handle* h, int dtype, int M, int N, int K, const void* a, const void* w,
                   const float* bias, int epilogue, const void* residual, void* out, void* stream) {
-  if (!h || !a || !w || !bias || !out || M < 0 || N < 1 || K < 1) return VIT_ERR_INVALID_ARG;
+  return vit_op_linear_tiled(h, dtype, M, N, K, a, w, bias, epilogue, residual, out, VIT_TILING_AUTO, stream);
+}
+
+int vit_op_linear_tiled(vit_handle* h, int dtype, int M, int N, int K, const void* a, const void* w,
+                        const float* bias, int epilogue, const void* residual, void* out, int tiling,
+                        void* stream) {
+  if (!h || !a || !w || !bias || !out || M < 0 || N < 1 || K < 1 || !on_own_device(h)) return VIT_ERR_INVALID_ARG;
+  if (tiling < VIT_TILING_AUTO || tiling > VIT_TILING_PAIR_256x256) return VIT_ERR_INVALID_ARG;
+  if (dtype != VIT_BF16 && tiling != VIT_TILING_AUTO) return VIT_ERR_INVALID_ARG;
   if (epilogue < 0 || epilogue > 2 || (epilogue == 2 && !residual)) return VIT_ERR_INVALID_ARG;
   if (misaligned(a) || misaligned(w) || misaligned(out) || misaligned(bias) || misaligned(residual))
     return VIT_ERR_INVALID_ARG;
   LinearArgs p{};
   p.M = M; p.N = N; p.K = K; p.a = a; p.lda = K; p.w = w; p.ldw = K; p.bias = bias;
   p.epilogue = epilogue; p.residual = residual; p.out = out; p.ldo = N;
+  p.tiling = tiling;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (dtype == VIT_BF16) {
     if (K % 8 || N % 8) return VIT_ERR_INVALID_ARG;
@@ -562,7 +584,7 @@ int vit_op_linear(vit_handle* h, int dtype, int M, int N, int K, const void* a, 
 
 int vit_op_attention(vit_handle* h, int dtype, int images, int T, int heads, int d, const void* qkv,
                      void* out, void* stream) {
-  if (!h || !qkv || !out || images < 0 || T < 1 || T > 512 || heads < 1 || d < 1) return VIT_ERR_INVALID_ARG;
+  if (!h || !qkv || !out || images < 0 || T < 1 || T > 512 || heads < 1 || d < 1 || !on_own_device(h)) return VIT_ERR_INVALID_ARG;
   if (misaligned(qkv) || misaligned(out)) return VIT_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (dtype == VIT_BF16) {

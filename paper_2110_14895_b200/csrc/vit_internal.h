@@ -5,6 +5,7 @@
 #include <stdint.h>
 #include <stddef.h>
 #include <atomic>
+#include <mutex>
 #include <vector>
 
 #include "../../include/vit.h"
@@ -35,7 +36,11 @@ struct LinearArgs {
   int n_patches;          // EPI_BIAS_POS
   void* out;              // activation type, row stride ldo
   int ldo;
+  int tiling;             // bf16 tensor-core kernel: TILING_AUTO (shape-only cost model) or a forced tiling
 };
+
+// Tilings of the tensor-core linear kernel (LinearArgs::tiling).
+enum Tiling : int { TILING_AUTO = 0, TILING_128x128 = 1, TILING_128x256 = 2, TILING_PAIR_256x256 = 3 };
 
 struct LayerWeights {
   const float *ln1_g, *ln1_b, *bqkv, *bo, *ln2_g, *ln2_b, *b1, *b2;
@@ -46,6 +51,7 @@ struct ProfRecord { cudaEvent_t begin, end; int cls; };
 
 struct Handle {
   vit_config cfg;
+  int device;                        // the CUDA device the handle was created on
   int T, n_patches, d, patch_k, patch_k_pad;
   size_t act_bytes;                  // bytes of one activation element
   void* dev_blob;                    // every parameter, one allocation
@@ -55,7 +61,8 @@ struct Handle {
   LayerWeights* layers;              // host array [L]
   const float *lnf_g, *lnf_b, *head_b;
   const void* head_W;                // [classes, H]
-  int* dev_status;                   // device status word (0 = ok)
+  int* dev_status;                   // device: [0] status word (0 = ok), [1] snapshot slot of vit_check_status
+  std::mutex status_mutex;
   std::atomic<uint64_t> launches;
   bool profiling;                    // event pair around every launch (single-threaded use)
   std::vector<ProfRecord> prof;
@@ -93,7 +100,27 @@ cudaError_t launch_head_static(const void* tokens, const float* g, const float* 
                                int H, int classes, bool act_bf16, cudaStream_t s);
 
 cudaError_t launch_wait_probe(long long limit_cycles, int* dev_status, cudaStream_t s);
+// *snapshot = atomic exchange of *status with 0, on stream s
+cudaError_t launch_status_take(int* status, int* snapshot, cudaStream_t s);
 
 bool tc_gemm_init();   // resolves the driver's tensor-map encoder; false if unavailable
+
+// Function attributes (the opt-in to more than 48 KB of dynamic shared memory) and the SM count
+// belong to a device, not to the process: each kernel instantiation keeps one bit per device.
+struct PerDeviceFlag {
+  std::atomic<uint64_t> mask{0};
+};
+template <typename Kernel>
+inline cudaError_t ensure_dynamic_smem(PerDeviceFlag& done, Kernel kernel, int bytes) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const bool tracked = dev >= 0 && dev < 64;
+  if (tracked && (done.mask.load(std::memory_order_acquire) >> dev & 1)) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess && tracked) done.mask.fetch_or((uint64_t)1 << dev, std::memory_order_release);
+  return e;
+}
+int current_device_sm_count();   // SMs of the current device (cached per device); 0 on error
 
 }  // namespace vit

@@ -193,17 +193,22 @@ def test_huge14_batch128_single_stage_equals_eight_stages_and_oracle():
     m.close()
 
 
-def test_huge14_microbatch_sweep_on_streams_is_consistent():
-    """Microbatch sizes through a 4-stage partition on streams: every size gives finite logits
-    that agree with the batch-of-one result within the bf16 tolerance (tile shapes may differ
-    between sizes, so bit equality is not required)."""
+def test_huge14_microbatch_sweep_every_size_matches_oracle():
+    """The microbatch sweep in full: 256 images of ViT-H/14 through four stages of eight layers,
+    microbatch sizes 1 ... 256 on min(4, 256/size) streams.  Every size is compared with the
+    oracle on images that are the first or the last of a microbatch at that size (image 0 and
+    255 at every size, 63|64 and 127|128 at sizes up to 64 and 128).  Tile shapes differ between
+    sizes, so the sizes are not required to agree bit for bit; their largest mutual difference is
+    printed."""
     shape = vitgen.preset("huge14")
-    vit, m, params = _model(shape, _vit().VIT_BF16, 32)
-    B = 32
+    vit, m, params = _model(shape, _vit().VIT_BF16, 256)
+    B = 256
     pix = vitgen.make_pixels(shape, B, seed=0)
     dp = torch.from_numpy(pix).cuda()
-    ref = None
-    for mb in (1, 2, 4, 8, 16, 32):
+    sample = [0, 63, 64, 127, 128, 255]
+    want = O.forward(params, shape, pix[sample])
+    first = None
+    for mb in (1, 2, 4, 8, 16, 32, 64, 128, 256):
         ns = min(4, B // mb)
         wss, streams, wsb = m.make_pipeline_buffers(mb, ns)
         logits = torch.full((B, shape.num_classes), float("nan"), dtype=torch.float32, device="cuda")
@@ -212,16 +217,15 @@ def test_huge14_microbatch_sweep_on_streams_is_consistent():
         for s in streams:
             m.check(s)
         got = logits.cpu().numpy()
-        assert np.isfinite(got).all()
-        if ref is None:
-            ref = got
-            want = O.forward(params, shape, pix[[0, 31]])
-            ok, msg = logits_within_tolerance(got[[0, 31]], want, 2e-2, 0.9995)
-            assert ok, msg
+        assert np.isfinite(got).all(), mb
+        ok, msg = logits_within_tolerance(got[sample], want, 2e-2, 0.9995)
+        assert ok, (mb, msg)
+        if first is None:
+            first = got
         else:
-            ok, msg = logits_within_tolerance(got, ref.astype(np.float64), 2e-2, 0.9995)
-            assert ok, (mb, msg)
-        del wss
+            print(f"microbatch {mb}: max |logit - logit at microbatch 1| = {np.abs(got - first).max():.3e}")
+        del wss, logits
+        torch.cuda.empty_cache()
     m.close()
 
 

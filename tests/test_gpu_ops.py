@@ -78,9 +78,25 @@ LINEAR_SHAPES = [
 @pytest.mark.parametrize("M,N,K", LINEAR_SHAPES)
 @pytest.mark.parametrize("epi", [0, 1, 2])
 def test_linear_bf16(ctx, M, N, K, epi):
+    _linear_case(ctx, M, N, K, epi, 0)
+
+
+# every tiling of the tensor-core kernel (128x128, 128x256, CTA pair 256x256) with every epilogue:
+# a ragged shape (partial tiles in M and N, K not a multiple of 64), a shape of several rounds of
+# the static schedule with an odd number of row tiles, and the fc1 / fc2 shapes of ViT-H at a
+# quarter batch (pair tiling is what the cost model picks there)
+TILED_SHAPES = [(300, 1000 // 8 * 8, 328), (129 * 37, 1280, 1280), (257 * 32, 5120, 1280), (257 * 32, 1280, 5120)]
+
+
+@pytest.mark.parametrize("M,N,K", TILED_SHAPES)
+@pytest.mark.parametrize("tiling", [1, 2, 3])
+@pytest.mark.parametrize("epi", [0, 1, 2])
+def test_linear_bf16_every_tiling(ctx, M, N, K, epi, tiling):
+    _linear_case(ctx, M, N, K, epi, tiling)
+
+
+def _linear_case(ctx, M, N, K, epi, tiling):
     vit, m = ctx
-    if epi != 0 and M * N * K > 3e9:
-        pytest.skip("large shapes checked with the plain epilogue only")
     rng = np.random.default_rng(M + 3 * N + 7 * K + epi)
     a, ar = _bf16(rng.normal(size=(M, K)))
     w, wr = _bf16(rng.normal(size=(N, K)) / np.sqrt(K))
@@ -92,7 +108,11 @@ def test_linear_bf16(ctx, M, N, K, epi):
         resp = out.data_ptr()
     else:
         resp = 0
-    vit.vit_op_linear(m.h, vit.VIT_BF16, M, N, K, a.data_ptr(), w.data_ptr(), bias.data_ptr(), epi, resp, out.data_ptr())
+    if tiling == 0:
+        vit.vit_op_linear(m.h, vit.VIT_BF16, M, N, K, a.data_ptr(), w.data_ptr(), bias.data_ptr(), epi, resp, out.data_ptr())
+    else:
+        vit.vit_op_linear_tiled(m.h, vit.VIT_BF16, M, N, K, a.data_ptr(), w.data_ptr(), bias.data_ptr(), epi, resp,
+                                out.data_ptr(), tiling)
     m.check()
     want = O.linear(ar, wr, br)
     if epi == 1:
@@ -135,7 +155,7 @@ def _oracle_attention(qkv, images, T, heads):
 
 
 @pytest.mark.parametrize("images,T,heads,d", [(1, 5, 2, 16), (2, 197, 3, 64), (3, 257, 2, 80), (1, 32, 1, 128),
-                                              (2, 33, 2, 64), (1, 16, 1, 32), (1, 300, 1, 96),
+                                              (2, 33, 2, 64), (1, 16, 1, 32), (1, 300, 1, 96), (1, 70, 2, 112),
                                               (2, 258, 1, 64), (1, 260, 2, 80), (2, 193, 2, 80), (1, 208, 1, 64),
                                               (1, 241, 1, 80), (1, 256, 2, 64)])
 @pytest.mark.parametrize("spread", [0.5, 4.0])

@@ -1,23 +1,25 @@
 // Fused multi-head self-attention on the 5th-generation tensor cores, for the sequence lengths
 // of ViT (T = 197 or 257 tokens; any T in [193,208] or [241,260]) and head sizes 64 and 80.
 //
-// One CTA per (image, head), two CTAs per SM.  K, V and one 128-query tile of Q are brought into
-// shared memory by TMA: columns [0,64) of the head as 128-byte-swizzled rows, columns [64,80)
-// (d = 80 only) as 32-byte-swizzled rows.  The same tiles serve as K-major operands (Q, K in
-// S = Q K^T) and as the N-major operand (V in O = P V).  Per query tile:
-//   S = Q K^T        tcgen05.mma, 128 x NK x d, accumulator in tensor memory (NK fp32 columns)
-//   softmax          8 warps, two threads per query row (each half of the keys): row max, exp2,
-//                    row sum, halves combined through shared memory; P is written back over S
-//                    as packed bf16 (tcgen05.st), so scores never leave the SM
-//   O = P V          tcgen05.mma with A = P from tensor memory, B = V from shared memory (for
-//                    d = 80, V is held as five 32-byte-swizzled blocks of 16 columns)
-//   epilogue         O / rowsum -> bf16 -> global
-// Keys beyond NK = 256 (the 257th token) are handled by the row's thread with plain FMAs on
-// copies of those K/V rows in shared memory.
-// Warps: 0-7 softmax/epilogue (warp w reads tensor-memory lanes 32 (w % 4) ...), 8 = TMA + MMA
-// issue + tensor-memory allocation.
-// The two resident CTAs overlap one's softmax with the other's loads and MMAs.
-// Every mbarrier wait is bounded; on expiry the CTA raises the device status word and leaves.
+// Persistent kernel, one CTA per SM, all 512 tensor-memory columns; a CTA walks over (image, head)
+// pairs with a static schedule.  Per head the 256 queries that fit two 128-row tiles are handled
+// by two softmax warpgroups side by side, one tile each, sharing one copy of K and V:
+//   TMA warp     K, V of the next head into the other of two shared-memory stages while this
+//                head is computed; Q (two tiles) as soon as the S products have read the old one.
+//                Columns [0,64) of the head are 128-byte-swizzled rows, columns [64,80) (d = 80)
+//                32-byte-swizzled rows; V for d = 80 is five 32-byte-swizzled 16-column blocks.
+//   MMA warp     per tile: S = Q K^T (tcgen05.mma, 128 x NKP x d, fp32 in tensor memory), later
+//                O = P V with A = P read from tensor memory and V as the N-major B operand,
+//                issued in two parts as P becomes ready.  The two tiles advance independently.
+//   softmax      2 x 4 warps, one thread per query row: row max, exp2, row sum; P is written back
+//                over S as packed bf16 (tcgen05.st), O lands in columns S no longer needs; then
+//                O / rowsum -> bf16 -> global.  While one warpgroup is in its exp2 phase the
+//                tensor core works for the other.
+//   helper warps the 257th token (ViT-H) on warp-level MMAs: its score column joins the row max
+//                and its probability is appended to P as one more 16-key step of P V (the rows
+//                of V behind it are zeroed); the 257th query row is computed start to finish.
+// Scores never leave the SM.  Every mbarrier wait is bounded; on expiry the CTA raises the device
+// status word, waits (bounded) for its copies and MMAs in flight, frees tensor memory and leaves.
 #include "vit_internal.h"
 #include "sm100_ptx.cuh"
 
@@ -29,12 +31,14 @@ namespace {
 
 using namespace ptx;
 
-constexpr int QT = 128;          // queries per tile = tensor-memory lanes
-constexpr int MAX_EXTRA = 4;     // keys beyond NK handled without the tensor cores
-constexpr int SOFTMAX_THREADS = 8 * 32;
-constexpr int NUM_THREADS = SOFTMAX_THREADS + 32;
-constexpr int MMA_WARP = 8;
-constexpr uint32_t TMEM_COLS = 256;
+constexpr int QT = 128;              // queries per tile = tensor-memory lanes
+constexpr int MAX_EXTRA = 4;         // tokens beyond 256 handled outside the two tiles
+constexpr int SOFTMAX_WARPS = 8;     // warps 0-3: tile 0, warps 4-7: tile 1
+constexpr int MMA_WARP = 8, TMA_WARP = 9, AUX_WARP0 = 10, AUX_WARPS = 4;
+constexpr int AUX_THREADS = AUX_WARPS * 32;
+constexpr int NUM_THREADS = (SOFTMAX_WARPS + 2 + AUX_WARPS) * 32;
+constexpr uint32_t TMEM_COLS = 512, TILE_COLS = 256;
+constexpr long long DRAIN_LIMIT_CYCLES = 1ll << 24;   // teardown after a failed wait: ~10 ms
 
 // Shared-memory matrix descriptors for TMA-written tiles whose rows are one swizzle span wide
 // (128 or 32 bytes); groups of 8 rows are 8 spans apart.  The same descriptor form serves a
@@ -61,363 +65,572 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&h);
 }
-__device__ __forceinline__ uint4 lds128(uint32_t a) {
-  uint4 u;
-  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(u.x), "=r"(u.y), "=r"(u.z), "=r"(u.w) : "r"(a));
-  return u;
+
+// warp-level tensor-core fragments for the helper warps (m16n8k16, bf16 operands, fp32 accumulate)
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t saddr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(saddr));
 }
-__device__ __forceinline__ float dot8(const uint4& a, const uint4& b, float acc) {
-  const __nv_bfloat162* ah = reinterpret_cast<const __nv_bfloat162*>(&a);
-  const __nv_bfloat162* bh = reinterpret_cast<const __nv_bfloat162*>(&b);
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const float2 x = __bfloat1622float2(ah[j]), y = __bfloat1622float2(bh[j]);
-    acc = fmaf(x.x, y.x, acc);
-    acc = fmaf(x.y, y.y, acc);
-  }
-  return acc;
+__device__ __forceinline__ void ldmatrix_x2(uint32_t (&r)[2], uint32_t saddr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0, %1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(saddr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t saddr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(saddr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, "
+      "{%8, %9}, {%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-struct AttnMaps { CUtensorMap q64, q16, kv64, kv16; };
+struct AttnMaps { CUtensorMap q64, q16, k64m, k64x, k16m, k16x; };
 
-// Tensor-memory columns (256 per CTA).  S occupies [0, NK).  The two threads of a row each own
-// half of the keys and overwrite S with P (bf16 pairs) only inside columns they have already
-// consumed themselves: half 0 walks its 32-key chunks upwards and packs P from column 0; half 1
-// walks its chunks downwards and packs P downwards from column NK.  O sits in between.
-template <int NK>
-struct TmemMap {
-  static constexpr int SPLIT = (NK / 64) * 32;              // keys [0, SPLIT) -> half 0, [SPLIT, NK) -> half 1
-  static constexpr int END1 = SPLIT + ((NK - SPLIT + 31) / 32) * 32;   // end of half 1's last (maybe partial) chunk
-  static constexpr uint32_t O_COL = SPLIT / 2;
-  // first P column of the 32-key chunk that starts at key c0
-  __host__ __device__ static constexpr uint32_t p_col(int c0) {
-    return c0 < SPLIT ? (uint32_t)(c0 / 2) : (uint32_t)(NK - 16 * ((END1 - 32 - c0) / 32 + 1));
-  }
-  // P columns of the 16 keys of MMA step ks
-  __host__ __device__ static constexpr uint32_t p_col_step(int ks) {
-    return 16 * ks < SPLIT ? (uint32_t)(8 * ks)
-                           : p_col(SPLIT + ((16 * ks - SPLIT) / 32) * 32) + (uint32_t)((((16 * ks - SPLIT) / 16) % 2) * 8);
-  }
-};
-
-template <int D, int NK>
+// Shared memory.  K and V hold NKP rows for the tensor core plus, for NKP = 256, 16 more rows
+// (tokens 256 ... 271 of the image: the extra tokens, then rows that are zeroed or never read).
+template <int D, int NKP>
 struct Smem {
   static constexpr bool TAIL = D > 64;                 // columns [64, D) live in the 32-byte part
-  static constexpr uint32_t KA = NK * 128, QA = QT * 128;
-  static constexpr uint32_t KB = TAIL ? NK * 32 : 0, QB = TAIL ? QT * 32 : 0;
-  static constexpr uint32_t VBYTES = NK * D * 2;       // D = 64: one 128-byte-swizzled tile;
-                                                       // D = 80: five 32-byte-swizzled 16-column blocks
-  static constexpr uint32_t OFF_KA = 0, OFF_QA = KA, OFF_V = KA + QA;
-  static constexpr uint32_t OFF_KB = OFF_V + VBYTES, OFF_QB = OFF_KB + KB;
-  static constexpr uint32_t OFF_XK = OFF_QB + QB;      // extra K rows, plain [MAX_EXTRA][D]
-  static constexpr uint32_t OFF_XV = OFF_XK + MAX_EXTRA * D * 2;
-  static constexpr uint32_t OFF_RED = OFF_XV + MAX_EXTRA * D * 2;   // float [2 halves][QT] row max, then [2][QT] row sum
-  static constexpr uint32_t OFF_SX = OFF_RED + 4 * QT * 4;          // float [2 tiles][MAX_EXTRA][QT] extra-key scores
-  static constexpr uint32_t OFF_BARS = OFF_SX + 2 * MAX_EXTRA * QT * 4;
-  static constexpr uint32_t BYTES = OFF_BARS + 128 + 1024 /*alignment slack*/;
-  static constexpr uint32_t KV_TX = KA + KB + VBYTES, Q_TX = QA + QB;
+  static constexpr int XR = NKP == 256 ? 16 : 0;
+  static constexpr int KR = NKP + XR;                  // rows of the K and V tiles
+  static constexpr uint32_t KA = KR * 128, KB = TAIL ? KR * 32 : 0;
+  static constexpr uint32_t VBLK = KR * 32;            // d = 80: one 16-column block of V
+  static constexpr uint32_t VBYTES = TAIL ? (D / 16) * VBLK : KR * 128;
+  static constexpr uint32_t OFF_KA = 0, OFF_KB = KA, OFF_V = KA + KB;
+  static constexpr uint32_t STAGE = KA + KB + VBYTES;  // one head's K and V; two stages
+  static constexpr uint32_t OFF_QA = 2 * STAGE;        // two tiles of 128 x 128 B
+  static constexpr uint32_t OFF_QB = OFF_QA + 2 * QT * 128;
+  static constexpr uint32_t OFF_SX = OFF_QB + (TAIL ? 2 * QT * 32 : 0);   // float [2][MAX_EXTRA][256]
+  static constexpr uint32_t OFF_QX = OFF_SX + 2 * MAX_EXTRA * 256 * 4;    // bf16 [8][D]: Q rows 256 ... 263
+  static constexpr uint32_t OFF_SC = OFF_QX + 8 * D * 2;                  // float [MAX_EXTRA][XS]: their scores, then probabilities
+  static constexpr int XS = 272;
+  static constexpr uint32_t OFF_INV = OFF_SC + MAX_EXTRA * XS * 4;        // float [MAX_EXTRA]: 1 / row sum
+  static constexpr uint32_t OFF_BARS = OFF_INV + 16;
+  static constexpr uint32_t BYTES = OFF_BARS + 256 + 1024 /*alignment slack*/;
+  static constexpr uint32_t KV_TX = STAGE, Q_TX = 2 * QT * (TAIL ? 160 : 128);
+  // Tensor memory of one tile (256 columns).  S occupies [0, NKP) and is consumed in 32-column
+  // chunks.  P (bf16 pairs, 8 columns per 16 keys) overwrites columns that have been read: keys
+  // 0 ... 191 go to [0, 96), the remaining keys to [192, 224), the extra keys to [224, 232).  O is
+  // accumulated in [96, 96 + D), free once the first six chunks of S have been read, so that
+  // the first twelve 16-key steps of P V can run while the last chunks are still being worked on.
+  static constexpr int KLO = 12;                       // 16-key steps in the first part of P V
+  static constexpr uint32_t P_HI_COL = 192, PX_COL = 224, O_COL = 96;
+  __host__ __device__ static constexpr uint32_t p_col(int kstep) {
+    return kstep < KLO ? (uint32_t)(8 * kstep) : P_HI_COL + (uint32_t)(8 * (kstep - KLO));
+  }
+  static_assert(O_COL + D <= P_HI_COL && NKP > 16 * KLO && NKP <= 256, "tensor-memory map");
+  static_assert(BYTES <= 227 * 1024, "shared memory");
+  static_assert(STAGE % 1024 == 0 && KA % 1024 == 0 && OFF_V % 256 == 0 && (TAIL || OFF_V % 1024 == 0), "alignment");
 };
 
-template <int D, int NK>
-__global__ void __launch_bounds__(NUM_THREADS, 2)
+enum Bar : int {
+  KV_FULL0 = 0, KV_FULL1, KV_FREE0, KV_FREE1, Q_FULL, Q_FREE, S_READY0, S_READY1, PL_READY0, PL_READY1,
+  P_READY0, P_READY1, O_READY0, O_READY1, T_FREE0, T_FREE1, SX_READY, VZ_READY0, VZ_READY1, AUX_SYNC,
+  DRAIN, NUM_BARS
+};
+
+template <int D, int NKP>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
 attention_tc_kernel(const __grid_constant__ AttnMaps maps, const bf16* __restrict__ qkv,
-                    bf16* __restrict__ out, int T, int heads, int* dev_status) {
-  using L = Smem<D, NK>;
+                    bf16* __restrict__ out, int T, int heads, int total_heads, int* dev_status) {
+  using L = Smem<D, NKP>;
   constexpr int CH = D / 8;                      // 16-byte chunks per row
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sb = smem_u32(smem);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BARS);
-  const uint32_t kv_full = smem_u32(&bars[0]);   // K, V landed                 (TMA bytes)
-  const uint32_t q_full = smem_u32(&bars[1]);    // Q tile landed               (TMA bytes)
-  const uint32_t s_ready = smem_u32(&bars[2]);   // S complete in tensor memory (MMA commit)
-  const uint32_t p_ready = smem_u32(&bars[3]);   // P written                   (256 arrivals)
-  const uint32_t o_ready = smem_u32(&bars[4]);   // O complete                  (MMA commit)
-  const uint32_t t_free = smem_u32(&bars[5]);    // O read, tensor memory free  (256 arrivals)
-  const uint32_t q_read = smem_u32(&bars[6]);    // Q rows read by their threads (128 arrivals)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(&bars[7]);
+  auto bar = [&](int i) { return smem_u32(&bars[i]); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(&bars[NUM_BARS]);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int img = blockIdx.x / heads, hd = blockIdx.x % heads;
   const int H = heads * D;
   const size_t ld = (size_t)3 * H;
-  const bf16* base = qkv + (size_t)img * T * ld + (size_t)hd * D;   // Q of token 0 of this head
-  const int ntiles = (T + QT - 1) / QT;
-  const int n_extra = T > NK ? T - NK : 0;
+  const int n_x = T > 256 ? T - 256 : 0;         // tokens beyond the two tiles (NKP = 256 only)
+  const int n_iter = total_heads > (int)blockIdx.x ? (total_heads - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
 
   if (threadIdx.x == 0) {
     *abort_flag = 0;
-    mbar_init(kv_full, 1);
-    mbar_init(q_full, 1);
-    mbar_init(s_ready, 1);
-    mbar_init(p_ready, SOFTMAX_THREADS);
-    mbar_init(o_ready, 1);
-    mbar_init(t_free, SOFTMAX_THREADS);
-    mbar_init(q_read, QT);
+    mbar_init(bar(KV_FULL0), 1);
+    mbar_init(bar(KV_FULL1), 1);
+    mbar_init(bar(KV_FREE0), 1 + AUX_WARPS);     // PV products retired + helper warps done with K, V
+    mbar_init(bar(KV_FREE1), 1 + AUX_WARPS);
+    mbar_init(bar(Q_FULL), 1);
+    mbar_init(bar(Q_FREE), 1 + AUX_WARPS);       // S products retired + helper warps done with Q
+    for (int w = 0; w < 2; ++w) {
+      mbar_init(bar(S_READY0 + w), 1);
+      mbar_init(bar(PL_READY0 + w), 4);          // one arrival per softmax warp of the tile: keys 0 ... 191 of P
+      mbar_init(bar(P_READY0 + w), 4);           // the rest of P
+      mbar_init(bar(O_READY0 + w), 1);
+      mbar_init(bar(T_FREE0 + w), 4);
+      mbar_init(bar(VZ_READY0 + w), AUX_WARPS);
+    }
+    mbar_init(bar(SX_READY), AUX_WARPS);
+    mbar_init(bar(AUX_SYNC), AUX_WARPS);
+    mbar_init(bar(DRAIN), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == MMA_WARP) tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
   grid_dependency_wait();               // barrier set-up and allocation overlap the previous kernel's tail
   grid_launch_dependents();
-  // copies of the K and V rows of the keys beyond NK, as plain rows
-  for (int i = threadIdx.x; i < n_extra * CH * 2; i += NUM_THREADS) {
-    const int which = i / (n_extra * CH), j = i % (n_extra * CH), e = j / CH, c = j % CH;
-    const uint4 v = __ldg(reinterpret_cast<const uint4*>(base + (size_t)(NK + e) * ld + (which + 1) * H) + c);
-    *reinterpret_cast<uint4*>(smem + (which ? L::OFF_XV : L::OFF_XK) + (e * CH + c) * 16) = v;
-  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == MMA_WARP) {
-    // ------------------------------------------------------------------ TMA + MMA issuer
+  if (warp == TMA_WARP) {
+    // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      const int row_g = img * T;                 // global row of token 0
-      const int col_q = hd * D, col_k = H + hd * D, col_v = 2 * H + hd * D;
-      mbar_arrive_expect_tx(kv_full, L::KV_TX);
-      tma_load_2d(sb + L::OFF_KA, &maps.kv64, col_k, row_g, kv_full);
-      if (L::TAIL) {
-        tma_load_2d(sb + L::OFF_KB, &maps.kv16, col_k + 64, row_g, kv_full);
+      int armed_kv[2] = {0, 0}, armed_q = 0;     // how often each "full" barrier has been armed
+      bool ok = true;
+      for (int it = 0; it < n_iter && ok; ++it) {
+        const int work = (int)blockIdx.x + it * (int)gridDim.x;
+        const int img = work / heads, hd = work % heads;
+        const int row_g = img * T;               // global row of token 0
+        const int col_q = hd * D, col_k = H + hd * D, col_v = 2 * H + hd * D;
+        const int s = it & 1;
+        const uint32_t st = sb + (uint32_t)s * L::STAGE;
+        const uint32_t kf = bar(KV_FULL0 + s);
+        if (!mbar_wait(bar(KV_FREE0 + s), (uint32_t)(((it >> 1) & 1) ^ 1), abort_flag)) { ok = false; break; }
+        mbar_arrive_expect_tx(kf, L::KV_TX);
+        ++armed_kv[s];
+        tma_load_2d(st + L::OFF_KA, &maps.k64m, col_k, row_g, kf);
+        if (L::XR) tma_load_2d(st + L::OFF_KA + NKP * 128, &maps.k64x, col_k, row_g + NKP, kf);
+        if (L::TAIL) {
+          tma_load_2d(st + L::OFF_KB, &maps.k16m, col_k + 64, row_g, kf);
+          if (L::XR) tma_load_2d(st + L::OFF_KB + NKP * 32, &maps.k16x, col_k + 64, row_g + NKP, kf);
 #pragma unroll
-        for (int a = 0; a < D / 16; ++a)
-          tma_load_2d(sb + L::OFF_V + (uint32_t)(a * NK * 32), &maps.kv16, col_v + 16 * a, row_g, kv_full);
-      } else {
-        tma_load_2d(sb + L::OFF_V, &maps.kv64, col_v, row_g, kv_full);
+          for (int a = 0; a < D / 16; ++a) {
+            tma_load_2d(st + L::OFF_V + (uint32_t)a * L::VBLK, &maps.k16m, col_v + 16 * a, row_g, kf);
+            if (L::XR)
+              tma_load_2d(st + L::OFF_V + (uint32_t)a * L::VBLK + NKP * 32, &maps.k16x, col_v + 16 * a, row_g + NKP, kf);
+          }
+        } else {
+          tma_load_2d(st + L::OFF_V, &maps.k64m, col_v, row_g, kf);
+          if (L::XR) tma_load_2d(st + L::OFF_V + NKP * 128, &maps.k64x, col_v, row_g + NKP, kf);
+        }
+        if (!mbar_wait(bar(Q_FREE), (uint32_t)((it & 1) ^ 1), abort_flag)) { ok = false; break; }
+        mbar_arrive_expect_tx(bar(Q_FULL), L::Q_TX);
+        ++armed_q;
+#pragma unroll
+        for (int w = 0; w < 2; ++w) {
+          tma_load_2d(sb + L::OFF_QA + (uint32_t)w * QT * 128, &maps.q64, col_q, row_g + w * QT, bar(Q_FULL));
+          if (L::TAIL)
+            tma_load_2d(sb + L::OFF_QB + (uint32_t)w * QT * 32, &maps.q16, col_q + 64, row_g + w * QT, bar(Q_FULL));
+        }
       }
-      mbar_arrive_expect_tx(q_full, L::Q_TX);
-      tma_load_2d(sb + L::OFF_QA, &maps.q64, col_q, row_g, q_full);
-      if (L::TAIL) tma_load_2d(sb + L::OFF_QB, &maps.q16, col_q + 64, row_g, q_full);
-
-      bool ok = mbar_wait(kv_full, 0, abort_flag);
-      for (int t = 0; t < ntiles && ok; ++t) {
-        const uint32_t ph = (uint32_t)(t & 1);
-        if (!mbar_wait(q_full, ph, abort_flag)) break;
-        if (t > 0 && !mbar_wait(t_free, ph ^ 1, abort_flag)) break;
-        tc_fence_after();
+      if (*abort_flag) {
+        // a wait gave up somewhere: let the copies that were started land before the CTA leaves
+        volatile int never = 0;
+        for (int s = 0; s < 2; ++s)
+          if (armed_kv[s]) mbar_wait_limit(bar(KV_FULL0 + s), (uint32_t)((armed_kv[s] - 1) & 1), &never, DRAIN_LIMIT_CYCLES);
+        if (armed_q) mbar_wait_limit(bar(Q_FULL), (uint32_t)((armed_q - 1) & 1), &never, DRAIN_LIMIT_CYCLES);
+      }
+    }
+  } else if (warp == MMA_WARP) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      bool ok = true;
+      auto issue_s = [&](int w, uint32_t st) {
+        const uint32_t d_tmem = tmem_base + (uint32_t)w * TILE_COLS;
         // S = Q K^T: 16 columns of the head per step, 32 bytes further along the swizzled row
 #pragma unroll
         for (int k = 0; k < 4; ++k)
-          umma_bf16(tmem_base, make_desc_sw128(sb + L::OFF_QA) + (uint64_t)(2 * k),
-                    make_desc_sw128(sb + L::OFF_KA) + (uint64_t)(2 * k), idesc_bf16(NK, false), k > 0 ? 1u : 0u);
+          umma_bf16(d_tmem, make_desc_sw128(sb + L::OFF_QA + (uint32_t)w * QT * 128) + (uint64_t)(2 * k),
+                    make_desc_sw128(st + L::OFF_KA) + (uint64_t)(2 * k), idesc_bf16(NKP, false), k > 0 ? 1u : 0u);
         if (L::TAIL)
-          umma_bf16(tmem_base, make_desc_sw32(sb + L::OFF_QB), make_desc_sw32(sb + L::OFF_KB),
-                    idesc_bf16(NK, false), 1u);
-        umma_commit(s_ready);
-        if (t + 1 < ntiles) {
-          // next Q tile: the buffer is free once these MMAs have read it (and, when rows are
-          // also read by their threads for the extra keys, once they have)
-          if (!mbar_wait(s_ready, ph, abort_flag)) break;
-          if (n_extra > 0 && !mbar_wait(q_read, ph, abort_flag)) break;
-          mbar_arrive_expect_tx(q_full, L::Q_TX);
-          tma_load_2d(sb + L::OFF_QA, &maps.q64, col_q, row_g + (t + 1) * QT, q_full);
-          if (L::TAIL) tma_load_2d(sb + L::OFF_QB, &maps.q16, col_q + 64, row_g + (t + 1) * QT, q_full);
+          umma_bf16(d_tmem, make_desc_sw32(sb + L::OFF_QB + (uint32_t)w * QT * 32), make_desc_sw32(st + L::OFF_KB),
+                    idesc_bf16(NKP, false), 1u);
+        umma_commit(bar(S_READY0 + w));
+      };
+      const int ksteps = NKP / 16 + (n_x > 0 ? 1 : 0);
+      constexpr int KLO = L::KLO;
+      // O = P V: A = P in tensor memory (8 columns per 16 keys); B = V, 16 keys per step = two
+      // 8-row groups of the tile.  Issued in two parts, as the parts of P become ready.
+      auto issue_pv = [&](int w, uint32_t st, int k0, int k1) {
+        const uint32_t t0 = tmem_base + (uint32_t)w * TILE_COLS;
+#pragma unroll 1
+        for (int k = k0; k < k1; ++k) {
+          const uint64_t bdesc = L::TAIL ? make_desc_sw32_blocks(st + L::OFF_V + (uint32_t)(k * 512), L::VBLK)
+                                         : make_desc_sw128(st + L::OFF_V + (uint32_t)(k * 2048));
+          umma_bf16_ts(t0 + L::O_COL, t0 + L::p_col(k), bdesc, idesc_bf16(D, true), k > 0 ? 1u : 0u);
         }
-        if (!mbar_wait(p_ready, ph, abort_flag)) break;
-        tc_fence_after();
-        // O = P V: A = P in tensor memory (8 columns per 16 keys); B = V, 16 keys per step =
-        // two 8-row groups of the tile
+      };
+      // The two tiles advance independently: each walks S(h) -> first part of P V (h) -> rest of
+      // P V (h) -> S(h + 1) ..., and this thread issues whichever step has its inputs ready, so the
+      // warpgroups drift apart and one is in its exp2 phase while the tensor core serves the other.
+      // Q (one buffer) is released when both tiles have issued S(h), a K/V stage when both have
+      // issued all of P V (h).
+      int t_it[2] = {0, 0}, t_step[2] = {0, 0};      // per tile: head iteration; step 0 = S, 1 = PV first part, 2 = PV rest
+      int s_count[2] = {0, 0}, pv_count[2] = {0, 0}; // per stage: tiles that have issued S / all of PV
+      long long idle_since = clock64();
+      while ((t_it[0] < n_iter || t_it[1] < n_iter) && ok) {
+        bool progress = false;
 #pragma unroll
-        for (int k = 0; k < NK / 16; ++k) {
-          const uint64_t bdesc = L::TAIL ? make_desc_sw32_blocks(sb + L::OFF_V + (uint32_t)(k * 512), NK * 32)
-                                         : make_desc_sw128(sb + L::OFF_V + (uint32_t)(k * 2048));
-          umma_bf16_ts(tmem_base + TmemMap<NK>::O_COL, tmem_base + TmemMap<NK>::p_col_step(k), bdesc,
-                       idesc_bf16(D, true), k > 0 ? 1u : 0u);
+        for (int w = 0; w < 2; ++w) {
+          const int it = t_it[w];
+          if (it >= n_iter) continue;
+          const int s = it & 1;
+          const uint32_t st = sb + (uint32_t)s * L::STAGE;
+          const uint32_t hph = (uint32_t)(it & 1), kph = (uint32_t)((it >> 1) & 1);
+          if (t_step[w] == 0) {
+            if (!(mbar_try_wait(bar(KV_FULL0 + s), kph) && mbar_try_wait(bar(Q_FULL), hph) &&
+                  mbar_try_wait(bar(T_FREE0 + w), hph ^ 1)))
+              continue;
+            tc_fence_after();
+            issue_s(w, st);
+            if (++s_count[s] == 2) { s_count[s] = 0; umma_commit(bar(Q_FREE)); }
+            t_step[w] = 1;
+          } else if (t_step[w] == 1) {
+            if (!(mbar_try_wait(bar(VZ_READY0 + s), kph) && mbar_try_wait(bar(PL_READY0 + w), hph))) continue;
+            tc_fence_after();
+            issue_pv(w, st, 0, KLO);
+            t_step[w] = 2;
+          } else {
+            if (!mbar_try_wait(bar(P_READY0 + w), hph)) continue;
+            tc_fence_after();
+            issue_pv(w, st, KLO, ksteps);
+            umma_commit(bar(O_READY0 + w));
+            if (++pv_count[s] == 2) { pv_count[s] = 0; umma_commit(bar(KV_FREE0 + s)); }
+            t_step[w] = 0;
+            t_it[w] = it + 1;
+          }
+          progress = true;
         }
-        umma_commit(o_ready);
+        if (progress) {
+          idle_since = clock64();
+        } else if (*abort_flag || clock64() - idle_since > WAIT_LIMIT_CYCLES) {
+          *abort_flag = 1;
+          ok = false;
+        }
+      }
+      if (*abort_flag) {
+        volatile int never = 0;
+        umma_commit(bar(DRAIN));                 // products issued so far retire before tensor memory is freed
+        mbar_wait_limit(bar(DRAIN), 0, &never, DRAIN_LIMIT_CYCLES);
       }
     }
-  } else {
+  }
+  else if (warp < SOFTMAX_WARPS) {
     // ------------------------------------------------------------------ softmax + epilogue
-    const int quarter = warp & 3, half = warp >> 2;
-    const int row = quarter * 32 + lane;                    // tensor-memory lane = query row of the tile
-    const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    const int wg = warp >> 2, quarter = warp & 3;
+    const int tok = wg * QT + quarter * 32 + lane;          // token of this thread's query row
+    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)wg * TILE_COLS;
+    const bool warp_active = wg * QT + quarter * 32 < T;    // any valid row in this warp
+    const int kmax = T < NKP ? T : NKP;                     // keys the tensor core covers
     const float sl2 = 1.4426950408889634f / sqrtf((float)D);   // log2(e) / sqrt(d)
-    using TM = TmemMap<NK>;
-    constexpr int SPLIT = TM::SPLIT;
-    constexpr uint32_t O_COL = TM::O_COL;
-    const int k_begin = half ? SPLIT : 0, k_end = half ? NK : SPLIT;
-    float* red = reinterpret_cast<float*>(smem + L::OFF_RED);     // [0..1][QT] max, [2..3][QT] sum
-    float* sx = reinterpret_cast<float*>(smem + L::OFF_SX);       // [tile & 1][MAX_EXTRA][QT]
-    auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(1 + quarter) : "memory"); };
+    constexpr int NCH = (NKP + 31) / 32;                    // 32-key chunks of S (the last may be partial)
+    const float* sx_all = reinterpret_cast<const float*>(smem + L::OFF_SX);
     bool ok = true;
-
-    // Scores of the keys beyond NK for tile `tt` (half 0 only), by hand: the row of Q is read back
-    // from the swizzled tile, the K rows are plain copies.  Results go to shared memory for both
-    // halves; arrives on q_read.
-    auto extra_scores = [&](int tt) -> bool {
-      if (n_extra == 0 || half != 0) return true;
-      if (!mbar_wait(q_full, (uint32_t)(tt & 1), abort_flag)) return false;
-      if (tt * QT + quarter * 32 < T) {
-        uint4 q[CH];
-#pragma unroll
-        for (int c = 0; c < 8; ++c) q[c] = lds128(sb + L::OFF_QA + (uint32_t)(row * 128 + ((c ^ (row & 7)) << 4)));
-#pragma unroll
-        for (int c = 8; c < CH; ++c)
-          q[c] = lds128(sb + L::OFF_QB + (uint32_t)(row * 32 + (((c - 8) ^ ((row >> 2) & 1)) << 4)));
-#pragma unroll
-        for (int e = 0; e < MAX_EXTRA; ++e) {
-          if (e < n_extra) {
-            float acc = 0.f;
-#pragma unroll
-            for (int c = 0; c < CH; ++c) acc = dot8(q[c], lds128(sb + L::OFF_XK + (uint32_t)((e * CH + c) * 16)), acc);
-            sx[((tt & 1) * MAX_EXTRA + e) * QT + row] = acc;
-          }
-        }
-      }
-      mbar_arrive(q_read);
-      return true;
-    };
-    ok = extra_scores(0);
-
-    for (int t = 0; t < ntiles && ok; ++t) {
-      const uint32_t ph = (uint32_t)(t & 1);
-      const bool warp_active = t * QT + quarter * 32 < T;   // any valid row in this warp
-      const float* sxt = sx + (t & 1) * MAX_EXTRA * QT;
-      if (!mbar_wait(s_ready, ph, abort_flag)) { ok = false; break; }
+    for (int it = 0; it < n_iter && ok; ++it) {
+      const int work = (int)blockIdx.x + it * (int)gridDim.x;
+      const int img = work / heads, hd = work % heads;
+      const uint32_t hph = (uint32_t)(it & 1);
+      const float* sxh = sx_all + (it & 1) * MAX_EXTRA * 256;
+      if (!mbar_wait(bar(S_READY0 + wg), hph, abort_flag)) { ok = false; break; }
+      if (n_x > 0 && !mbar_wait(bar(SX_READY), hph, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      float msl = 0.f;
-      if (warp_active) {
-        // pass 1: maximum over this half's keys
-        float m = -INFINITY;
-        if (half == 0) {
-#pragma unroll
-          for (int e = 0; e < MAX_EXTRA; ++e)
-            if (e < n_extra) m = fmaxf(m, sxt[e * QT + row]);
-        }
-#pragma unroll 1
-        for (int c0 = k_begin; c0 < k_end; c0 += 32) {
-          uint32_t r[32];
-          tmem_ld32(lane_addr + (uint32_t)c0, r);      // the last chunk may run past NK: masked below
-          tmem_ld_wait();
-          if (c0 + 32 <= T && c0 + 32 <= NK) {
-            float m2[2] = {m, m};
-#pragma unroll
-            for (int j = 0; j < 32; j += 4) {
-              asm("max.f32 %0, %0, %1, %2;" : "+f"(m2[0]) : "f"(__uint_as_float(r[j])), "f"(__uint_as_float(r[j + 1])));
-              asm("max.f32 %0, %0, %1, %2;" : "+f"(m2[1]) : "f"(__uint_as_float(r[j + 2])), "f"(__uint_as_float(r[j + 3])));
-            }
-            m = fmaxf(m2[0], m2[1]);
-          } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (c0 + j < T && c0 + j < NK) m = fmaxf(m, __uint_as_float(r[j]));
-          }
-        }
-        red[half * QT + row] = m;
-      }
-      pair_sync();
       float l = 0.f;
       if (warp_active) {
-        msl = fmaxf(red[row], red[QT + row]) * sl2;
-        // pass 2: p = exp2((s - m) * sl2), partial row sum, P (bf16) back into tensor memory
-        // (half 0 upwards, half 1 downwards: see TmemMap)
-        const int nchunks = (k_end - k_begin + 31) / 32;
-#pragma unroll 1
-        for (int i = 0; i < nchunks; ++i) {
-          const int c0 = half ? k_begin + 32 * (nchunks - 1 - i) : k_begin + 32 * i;
-          uint32_t r[32];
-          tmem_ld32(lane_addr + (uint32_t)c0, r);
-          tmem_ld_wait();
+        // pass 1: row maximum, two 32-column loads per wait (the reduction is short; what counts
+        // is the latency of the tensor-memory loads)
+        float m = -INFINITY;
+#pragma unroll
+        for (int e = 0; e < MAX_EXTRA; ++e)
+          if (e < n_x) m = fmaxf(m, sxh[e * 256 + tok]);
+        uint32_t r[2][32];
+#pragma unroll
+        for (int i = 0; i < NCH; i += 2) {
+          tmem_ld32(taddr + (uint32_t)(32 * i), r[0]);
+          if (i + 1 < NCH) tmem_ld32(taddr + (uint32_t)(32 * (i + 1)), r[1]);
+          tmem_ld_wait_for(r[0]);
+          if (i + 1 < NCH) tmem_ld_wait_for(r[1]);
+#pragma unroll
+          for (int h2 = 0; h2 < 2; ++h2) {
+            if (i + h2 >= NCH) continue;
+            const uint32_t (&c)[32] = r[h2];
+            const int c0 = 32 * (i + h2);
+            if (c0 + 32 <= kmax) {
+              float m2[2] = {m, m};
+#pragma unroll
+              for (int j = 0; j < 32; j += 4) {
+                asm("max.f32 %0, %0, %1, %2;" : "+f"(m2[0]) : "f"(__uint_as_float(c[j])), "f"(__uint_as_float(c[j + 1])));
+                asm("max.f32 %0, %0, %1, %2;" : "+f"(m2[1]) : "f"(__uint_as_float(c[j + 2])), "f"(__uint_as_float(c[j + 3])));
+              }
+              m = fmaxf(m2[0], m2[1]);
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (c0 + j < kmax) m = fmaxf(m, __uint_as_float(c[j]));
+            }
+          }
+        }
+        const float msl = m * sl2;
+        // pass 2: p = exp2((s - m) * sl2), row sum, P (bf16 pairs) back into tensor memory over
+        // columns this thread has already read (see the tensor-memory map).  The load of chunk
+        // i + 1 is in flight while chunk i is worked on.  After six chunks (keys 0 ... 191) the
+        // tensor core is told to start on O.
+        float2 l2 = make_float2(0.f, 0.f);
+        const float2 sl2v = make_float2(sl2, sl2), nmsl = make_float2(-msl, -msl);
+        tmem_ld32(taddr, r[0]);
+#pragma unroll
+        for (int i = 0; i < NCH; ++i) {
+          tmem_ld_wait_for(r[i & 1]);
+          if (i + 1 < NCH) tmem_ld32(taddr + (uint32_t)(32 * (i + 1)), r[(i + 1) & 1]);
+          const uint32_t (&c)[32] = r[i & 1];
           uint32_t pk[16];
-          if (c0 + 32 <= T && c0 + 32 <= NK) {
-            float l2[2] = {0.f, 0.f};
+          if (32 * i + 32 <= kmax) {
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
-              const float p0 = ex2_approx(fmaf(__uint_as_float(r[2 * j]), sl2, -msl));
-              const float p1 = ex2_approx(fmaf(__uint_as_float(r[2 * j + 1]), sl2, -msl));
-              l2[0] += p0;
-              l2[1] += p1;
-              pk[j] = pack_bf16(p0, p1);
+              const float2 x = __ffma2_rn(make_float2(__uint_as_float(c[2 * j]), __uint_as_float(c[2 * j + 1])), sl2v, nmsl);
+              const float2 pp = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+              l2 = __fadd2_rn(l2, pp);
+              pk[j] = pack_bf16(pp.x, pp.y);
             }
-            l += l2[0] + l2[1];
           } else {
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
-              const int k0 = c0 + 2 * j;
-              const float p0 = (k0 < T && k0 < NK) ? ex2_approx(fmaf(__uint_as_float(r[2 * j]), sl2, -msl)) : 0.f;
-              const float p1 = (k0 + 1 < T && k0 + 1 < NK) ? ex2_approx(fmaf(__uint_as_float(r[2 * j + 1]), sl2, -msl)) : 0.f;
-              l += p0 + p1;
+              const int k0 = 32 * i + 2 * j;
+              const float p0 = k0 < kmax ? ex2_approx(fmaf(__uint_as_float(c[2 * j]), sl2, -msl)) : 0.f;
+              const float p1 = k0 + 1 < kmax ? ex2_approx(fmaf(__uint_as_float(c[2 * j + 1]), sl2, -msl)) : 0.f;
+              l2.x += p0;
+              l2.y += p1;
               pk[j] = pack_bf16(p0, p1);
             }
           }
-          tmem_st16(lane_addr + TM::p_col(c0), pk);
+          if (32 * i + 32 <= NKP) {
+            tmem_st16(taddr + L::p_col(2 * i), pk);
+          } else {                                   // NKP = 208: the last chunk holds 16 keys
+            uint32_t part[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) part[j] = pk[j];
+            tmem_st8(taddr + L::p_col(2 * i), part);
+          }
+          if (i == 5) {                              // keys 0 ... 191 of P are in place
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(PL_READY0 + wg));
+          }
         }
-        red[(2 + half) * QT + row] = l;
+        l = l2.x + l2.y;
+        if (n_x > 0) {
+          // the extra keys' probabilities: one more 16-key step of P (keys 256 ... 271)
+          float px[MAX_EXTRA];
+#pragma unroll
+          for (int e = 0; e < MAX_EXTRA; ++e) {
+            px[e] = e < n_x ? ex2_approx(fmaf(sxh[e * 256 + tok], sl2, -msl)) : 0.f;
+            l += px[e];
+          }
+          const uint32_t xp[8] = {pack_bf16(px[0], px[1]), pack_bf16(px[2], px[3]), 0u, 0u, 0u, 0u, 0u, 0u};
+          tmem_st8(taddr + L::PX_COL, xp);
+        }
         tmem_st_wait();
+      } else {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(PL_READY0 + wg));
       }
       tc_fence_before();
-      mbar_arrive(p_ready);
-      // while the tensor core runs P V: the extra keys' scores of the next tile
-      if (t + 1 < ntiles && !extra_scores(t + 1)) { ok = false; break; }
-      // epilogue: O (+ the hand-computed keys' share) / l -> bf16 -> global; this half's columns
-      if (!mbar_wait(o_ready, ph, abort_flag)) { ok = false; break; }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(P_READY0 + wg));
+      // epilogue: O / l -> bf16 -> global
+      if (!mbar_wait(bar(O_READY0 + wg), hph, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      pair_sync();                                          // both partial sums are in shared memory
-      constexpr int G0 = (D / 16 + 1) / 2;                  // 16-column groups [0, G0) -> half 0, the rest -> half 1
-      const int g_begin = half ? G0 : 0, g_end = half ? D / 16 : G0;
-      uint32_t oreg[G0 * 16];
+      uint32_t o[D];
       if (warp_active) {
 #pragma unroll
-        for (int g = 0; g < G0; ++g)
-          if (g_begin + g < g_end)
-            tmem_ld16(lane_addr + O_COL + (uint32_t)((g_begin + g) * 16), *reinterpret_cast<uint32_t(*)[16]>(&oreg[g * 16]));
+        for (int g = 0; g < D / 16; ++g)
+          tmem_ld16(taddr + L::O_COL + (uint32_t)(g * 16), *reinterpret_cast<uint32_t(*)[16]>(&o[g * 16]));
         tmem_ld_wait();
       }
       tc_fence_before();
-      mbar_arrive(t_free);               // the next tile's S may overwrite tensor memory now
-      const int tok = t * QT + row;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(T_FREE0 + wg));   // the next head's S may overwrite this tile now
       if (warp_active && tok < T) {
-        l = red[2 * QT + row] + red[3 * QT + row];
-        float p_ex[MAX_EXTRA];
-#pragma unroll
-        for (int e = 0; e < MAX_EXTRA; ++e) {
-          p_ex[e] = e < n_extra ? ex2_approx(fmaf(sxt[e * QT + row], sl2, -msl)) : 0.f;
-          l += p_ex[e];
-        }
         const float inv = 1.0f / l;
         uint4* orow = reinterpret_cast<uint4*>(out + ((size_t)img * T + tok) * H + (size_t)hd * D);
 #pragma unroll
-        for (int g = 0; g < G0; ++g) {
-          if (g_begin + g < g_end) {
+        for (int c = 0; c < CH; ++c) {
+          uint4 w;
+          w.x = pack_bf16(__uint_as_float(o[8 * c + 0]) * inv, __uint_as_float(o[8 * c + 1]) * inv);
+          w.y = pack_bf16(__uint_as_float(o[8 * c + 2]) * inv, __uint_as_float(o[8 * c + 3]) * inv);
+          w.z = pack_bf16(__uint_as_float(o[8 * c + 4]) * inv, __uint_as_float(o[8 * c + 5]) * inv);
+          w.w = pack_bf16(__uint_as_float(o[8 * c + 6]) * inv, __uint_as_float(o[8 * c + 7]) * inv);
+          orow[c] = w;
+        }
+      }
+    }
+  }
+  else if (warp >= AUX_WARP0) {
+    // ------------------------------------------------------------------ helper warps
+    const int j = threadIdx.x - AUX_WARP0 * 32;             // 0 ... AUX_THREADS - 1
+    const int aw = warp - AUX_WARP0;
+    const float sl2 = 1.4426950408889634f / sqrtf((float)D);
+    float* sx_all = reinterpret_cast<float*>(smem + L::OFF_SX);
+    float* sc = reinterpret_cast<float*>(smem + L::OFF_SC);
+    float* inv_l = reinterpret_cast<float*>(smem + L::OFF_INV);
+    const uint32_t qxb = sb + L::OFF_QX;
+    // fragment coordinates of this lane: ldmatrix row / 16-byte chunk offsets, mma row and column pair
+    const int lrow = (lane & 7) + 8 * ((lane >> 3) & 1), lchunk = lane >> 4;
+    const int g = lane >> 2, t2 = 2 * (lane & 3);
+    uint32_t aux_phase = 0;
+    bool ok = true;
+    // barrier among the helper warps (bounded like every other wait)
+    auto aux_sync = [&]() -> bool {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(AUX_SYNC));
+      const bool done = mbar_wait(bar(AUX_SYNC), aux_phase, abort_flag);
+      aux_phase ^= 1;
+      return done;
+    };
+    // shared-memory address of 16-byte chunk c of row r of V (st = stage base)
+    auto v_chunk = [&](uint32_t st, int r, int c) -> uint32_t {
+      return L::TAIL ? st + L::OFF_V + (uint32_t)((c >> 1) * L::VBLK + r * 32 + (((c & 1) ^ ((r >> 2) & 1)) << 4))
+                     : st + L::OFF_V + (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4));
+    };
+    // Fragment addresses for the warp-level MMAs, k-step ks (16 head columns): this lane's row of a
+    // 16-row A tile that starts at row0 (a multiple of 16), and of an 8-row B tile (brow0 a multiple
+    // of 8).  main = the 128-byte-swizzled part (columns 0 ... 63), tail = the 32-byte part.
+    const uint32_t a_main = (uint32_t)(lrow * 128), a_tail = (uint32_t)(lrow * 32 + ((lchunk ^ ((lrow >> 2) & 1)) << 4));
+    const int hb = (lane >> 3) & 1, brow = lane & 7;
+    const uint32_t b_main = (uint32_t)(brow * 128), b_tail = (uint32_t)(brow * 32 + ((hb ^ ((brow >> 2) & 1)) << 4));
+    auto a_addr = [&](uint32_t main, uint32_t tail, int row0, int ks) -> uint32_t {
+      if (ks < 4) return main + (uint32_t)(row0 * 128) + a_main + (uint32_t)((((2 * ks + lchunk) ^ (lrow & 7))) << 4);
+      return tail + (uint32_t)(row0 * 32) + a_tail;
+    };
+    auto b_addr = [&](uint32_t main, uint32_t tail, int brow0, int ks) -> uint32_t {
+      if (ks < 4) return main + (uint32_t)(brow0 * 128) + b_main + (uint32_t)((((2 * ks + hb) ^ brow)) << 4);
+      return tail + (uint32_t)(brow0 * 32) + b_tail;
+    };
+    for (int it = 0; it < n_iter && ok; ++it) {
+      const int work = (int)blockIdx.x + it * (int)gridDim.x;
+      const int img = work / heads, hd = work % heads;
+      const int s = it & 1;
+      const uint32_t st = sb + (uint32_t)s * L::STAGE;
+      const uint32_t hph = (uint32_t)(it & 1), kph = (uint32_t)((it >> 1) & 1);
+      if (!mbar_wait(bar(KV_FULL0 + s), kph, abort_flag)) { ok = false; break; }
+      // rows of V behind the last token are multiplied by zero probabilities: make them zero too,
+      // so that whatever lies behind this image in memory cannot reach the result
+      for (int i = j; i < (L::KR - T) * CH; i += AUX_THREADS) {
+        const int r = T + i / CH, c = i % CH;
+        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(v_chunk(st, r, c)), "r"(0u) : "memory");
+      }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(VZ_READY0 + s));
+      if (!mbar_wait(bar(Q_FULL), hph, abort_flag)) { ok = false; break; }
+      if (n_x > 0) {
+        // scores of the extra keys for the 256 tile rows: [256 x d] . [d x 8] on warp-level MMAs,
+        // A = 16 rows of Q, B = rows 256 ... 263 of K (columns beyond the extra keys are not used)
+        float* sxh = sx_all + (it & 1) * MAX_EXTRA * 256;
+        uint32_t bk[D / 16][2];
 #pragma unroll
-            for (int q = 0; q < 2; ++q) {
-              const int c = (g_begin + g) * 2 + q;         // 16-byte chunk of the row
-              float o[8];
+        for (int ks = 0; ks < D / 16; ++ks) ldmatrix_x2(bk[ks], b_addr(st + L::OFF_KA, st + L::OFF_KB, 256, ks));
+#pragma unroll 1
+        for (int mt = aw; mt < 16; mt += AUX_WARPS) {
+          float c[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-              for (int j = 0; j < 8; ++j) o[j] = __uint_as_float(oreg[g * 16 + q * 8 + j]);
-              if (n_extra > 0) {
+          for (int ks = 0; ks < D / 16; ++ks) {
+            uint32_t a[4];
+            ldmatrix_x4(a, a_addr(sb + L::OFF_QA, sb + L::OFF_QB, mt * 16, ks));
+            mma_bf16(c, a, bk[ks][0], bk[ks][1]);
+          }
+          const int r0 = mt * 16 + g;
+          if (t2 < n_x) { sxh[t2 * 256 + r0] = c[0]; sxh[t2 * 256 + r0 + 8] = c[2]; }
+          if (t2 + 1 < n_x) { sxh[(t2 + 1) * 256 + r0] = c[1]; sxh[(t2 + 1) * 256 + r0 + 8] = c[3]; }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(bar(SX_READY));
+        mbar_arrive(bar(Q_FREE));
+      }
+      if (n_x > 0) {
+        // the extra query rows, start to finish, on warp-level MMAs.  Rows 256 ... 263 of Q as
+        // plain rows in shared memory (rows that are not extra queries are zero).
+        for (int i = j; i < 8 * CH; i += AUX_THREADS) {
+          const int e = i / CH, c = i % CH;
+          uint4 v = make_uint4(0u, 0u, 0u, 0u);
+          if (e < n_x) v = __ldg(reinterpret_cast<const uint4*>(qkv + ((size_t)img * T + 256 + e) * ld + (size_t)hd * D) + c);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(qxb + (uint32_t)(i * 16)), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+        }
+        if (!aux_sync()) { ok = false; break; }
+        // scores[key][e] = K[key] . Q[256 + e]
+        uint32_t bq[D / 16][2];
 #pragma unroll
-                for (int e = 0; e < MAX_EXTRA; ++e) {
-                  if (e < n_extra) {
-                    const uint4 va = lds128(sb + L::OFF_XV + (uint32_t)((e * CH + c) * 16));
-                    const __nv_bfloat162* vh = reinterpret_cast<const __nv_bfloat162*>(&va);
+        for (int ks = 0; ks < D / 16; ++ks)
+          ldmatrix_x2(bq[ks], qxb + (uint32_t)(((lane & 7) * CH + 2 * ks + ((lane >> 3) & 1)) * 16));
+        const int n_kt = (T + 15) / 16;                      // 16-key tiles
+#pragma unroll 1
+        for (int mt = aw; mt < n_kt; mt += AUX_WARPS) {
+          float c[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                      const float2 v2 = __bfloat1622float2(vh[j]);
-                      o[2 * j] = fmaf(p_ex[e], v2.x, o[2 * j]);
-                      o[2 * j + 1] = fmaf(p_ex[e], v2.y, o[2 * j + 1]);
-                    }
-                  }
-                }
-              }
-              uint4 w;
-              w.x = pack_bf16(o[0] * inv, o[1] * inv);
-              w.y = pack_bf16(o[2] * inv, o[3] * inv);
-              w.z = pack_bf16(o[4] * inv, o[5] * inv);
-              w.w = pack_bf16(o[6] * inv, o[7] * inv);
-              orow[c] = w;
+          for (int ks = 0; ks < D / 16; ++ks) {
+            uint32_t a[4];
+            ldmatrix_x4(a, a_addr(st + L::OFF_KA, st + L::OFF_KB, mt * 16, ks));
+            mma_bf16(c, a, bq[ks][0], bq[ks][1]);
+          }
+          const int k0 = mt * 16 + g;
+          if (t2 < n_x) { sc[t2 * L::XS + k0] = c[0]; sc[t2 * L::XS + k0 + 8] = c[2]; }
+          if (t2 + 1 < n_x) { sc[(t2 + 1) * L::XS + k0] = c[1]; sc[(t2 + 1) * L::XS + k0 + 8] = c[3]; }
+        }
+        if (!aux_sync()) { ok = false; break; }
+        // softmax of row e by one warp: probabilities (zero behind the last token) and 1 / row sum
+        for (int e = aw; e < n_x; e += AUX_WARPS) {
+          float* row = sc + e * L::XS;
+          float m = -INFINITY;
+          for (int key = lane; key < T; key += 32) m = fmaxf(m, row[key]);
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+          const float msl = m * sl2;
+          float lsum = 0.f;
+          for (int key = lane; key < n_kt * 16; key += 32) {
+            const float p = key < T ? ex2_approx(fmaf(row[key], sl2, -msl)) : 0.f;
+            row[key] = p;
+            lsum += p;
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
+          if (lane == 0) inv_l[e] = 1.0f / lsum;
+        }
+        if (!aux_sync()) { ok = false; break; }
+        // O[e][:] = P[e][:] V: A = probabilities (rows beyond the extra queries zero), B = V through
+        // transposing fragment loads; a warp owns pairs of 8-column tiles of the head
+#pragma unroll 1
+        for (int pr = aw; pr < CH / 2; pr += AUX_WARPS) {
+          float acc0[4] = {0.f, 0.f, 0.f, 0.f}, acc1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+          for (int kt = 0; kt < n_kt; ++kt) {
+            uint32_t a[4] = {0u, 0u, 0u, 0u};
+            if (g < n_x) {
+              const float2 p0 = *reinterpret_cast<const float2*>(sc + g * L::XS + kt * 16 + t2);
+              const float2 p1 = *reinterpret_cast<const float2*>(sc + g * L::XS + kt * 16 + 8 + t2);
+              a[0] = pack_bf16(p0.x, p0.y);
+              a[2] = pack_bf16(p1.x, p1.y);
             }
+            uint32_t b[4];
+            ldmatrix_x4_trans(b, v_chunk(st, kt * 16 + lrow, 2 * pr + lchunk));
+            mma_bf16(acc0, a, b[0], b[1]);
+            mma_bf16(acc1, a, b[2], b[3]);
+          }
+          if (g < n_x) {
+            const float inv = inv_l[g];
+            bf16* orow = out + ((size_t)img * T + 256 + g) * H + (size_t)hd * D + 16 * pr + t2;
+            *reinterpret_cast<uint32_t*>(orow) = pack_bf16(acc0[0] * inv, acc0[1] * inv);
+            *reinterpret_cast<uint32_t*>(orow + 8) = pack_bf16(acc1[0] * inv, acc1[1] * inv);
           }
         }
       }
+      if (!ok) break;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(KV_FREE0 + s));
     }
   }
 
   // ---------------------------------------------------------------------- teardown
   __syncwarp();
-  if (*abort_flag) __nanosleep(200000);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -445,10 +658,10 @@ bool encode_map(CUtensorMap* tm, const void* base, size_t rows, size_t cols, int
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D, int NK>
+template <int D, int NKP>
 cudaError_t launch_variant(const bf16* qkv, bf16* out, int images, int T, int heads, int* dev_status,
                            cudaStream_t s) {
-  using L = Smem<D, NK>;
+  using L = Smem<D, NKP>;
   if (!g_encode) {
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult q;
@@ -458,21 +671,28 @@ cudaError_t launch_variant(const bf16* qkv, bf16* out, int images, int T, int he
     g_encode = reinterpret_cast<EncodeTiledFn>(fn);
   }
   static PerDeviceFlag configured;
-  cudaError_t e = ensure_dynamic_smem(configured, attention_tc_kernel<D, NK>, (int)L::BYTES);
+  cudaError_t e = ensure_dynamic_smem(configured, attention_tc_kernel<D, NKP>, (int)L::BYTES);
   if (e != cudaSuccess) return e;
+  const int sms = current_device_sm_count();
+  if (sms < 1) return cudaErrorInvalidDevice;
   const size_t rows = (size_t)images * T, cols = (size_t)3 * heads * D;
+  const CUtensorMapSwizzle s128 = CU_TENSOR_MAP_SWIZZLE_128B, s32 = CU_TENSOR_MAP_SWIZZLE_32B;
   AttnMaps m;
-  if (!encode_map(&m.q64, qkv, rows, cols, 64, QT, CU_TENSOR_MAP_SWIZZLE_128B)) return cudaErrorInvalidValue;
-  if (!encode_map(&m.kv64, qkv, rows, cols, 64, NK, CU_TENSOR_MAP_SWIZZLE_128B)) return cudaErrorInvalidValue;
+  if (!encode_map(&m.q64, qkv, rows, cols, 64, QT, s128)) return cudaErrorInvalidValue;
+  if (!encode_map(&m.k64m, qkv, rows, cols, 64, NKP, s128)) return cudaErrorInvalidValue;
+  if (!encode_map(&m.k64x, qkv, rows, cols, 64, 16, s128)) return cudaErrorInvalidValue;
   if (D > 64) {
-    if (!encode_map(&m.q16, qkv, rows, cols, D - 64, QT, CU_TENSOR_MAP_SWIZZLE_32B)) return cudaErrorInvalidValue;
-    if (!encode_map(&m.kv16, qkv, rows, cols, D - 64, NK, CU_TENSOR_MAP_SWIZZLE_32B)) return cudaErrorInvalidValue;
+    if (!encode_map(&m.q16, qkv, rows, cols, 16, QT, s32)) return cudaErrorInvalidValue;
+    if (!encode_map(&m.k16m, qkv, rows, cols, 16, NKP, s32)) return cudaErrorInvalidValue;
+    if (!encode_map(&m.k16x, qkv, rows, cols, 16, 16, s32)) return cudaErrorInvalidValue;
   } else {
     m.q16 = m.q64;
-    m.kv16 = m.kv64;
+    m.k16m = m.k64m;
+    m.k16x = m.k64x;
   }
+  const int total = images * heads;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)(images * heads));
+  cfg.gridDim = dim3((unsigned)(total < sms ? total : sms));
   cfg.blockDim = dim3(NUM_THREADS);
   cfg.dynamicSmemBytes = L::BYTES;
   cfg.stream = s;
@@ -481,7 +701,7 @@ cudaError_t launch_variant(const bf16* qkv, bf16* out, int images, int T, int he
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, attention_tc_kernel<D, NK>, m, qkv, out, T, heads, dev_status);
+  return cudaLaunchKernelEx(&cfg, attention_tc_kernel<D, NKP>, m, qkv, out, T, heads, total, dev_status);
 }
 
 }  // namespace

@@ -9,8 +9,7 @@
 //                Columns [0,64) of the head are 128-byte-swizzled rows, columns [64,80) (d = 80)
 //                32-byte-swizzled rows; V for d = 80 is five 32-byte-swizzled 16-column blocks.
 //   MMA warp     per tile: S = Q K^T (tcgen05.mma, 128 x NKP x d, fp32 in tensor memory), later
-//                O = P V with A = P read from tensor memory and V as the N-major B operand,
-//                issued in two parts as P becomes ready.  The two tiles advance independently.
+//                O = P V with A = P read from tensor memory and V as the N-major B operand
 //   softmax      2 x 4 warps, one thread per query row: row max, exp2, row sum; P is written back
 //                over S as packed bf16 (tcgen05.st), O lands in columns S no longer needs; then
 //                O / rowsum -> bf16 -> global.  While one warpgroup is in its exp2 phase the
@@ -113,9 +112,8 @@ struct Smem {
   // Tensor memory of one tile (256 columns).  S occupies [0, NKP) and is consumed in 32-column
   // chunks.  P (bf16 pairs, 8 columns per 16 keys) overwrites columns that have been read: keys
   // 0 ... 191 go to [0, 96), the remaining keys to [192, 224), the extra keys to [224, 232).  O is
-  // accumulated in [96, 96 + D), free once the first six chunks of S have been read, so that
-  // the first twelve 16-key steps of P V can run while the last chunks are still being worked on.
-  static constexpr int KLO = 12;                       // 16-key steps in the first part of P V
+  // accumulated in [96, 96 + D).
+  static constexpr int KLO = 12;                       // 16-key steps whose P sits below O
   static constexpr uint32_t P_HI_COL = 192, PX_COL = 224, O_COL = 96;
   __host__ __device__ static constexpr uint32_t p_col(int kstep) {
     return kstep < KLO ? (uint32_t)(8 * kstep) : P_HI_COL + (uint32_t)(8 * (kstep - KLO));
@@ -126,7 +124,7 @@ struct Smem {
 };
 
 enum Bar : int {
-  KV_FULL0 = 0, KV_FULL1, KV_FREE0, KV_FREE1, Q_FULL, Q_FREE, S_READY0, S_READY1, PL_READY0, PL_READY1,
+  KV_FULL0 = 0, KV_FULL1, KV_FREE0, KV_FREE1, Q_FULL, Q_FREE, S_READY0, S_READY1,
   P_READY0, P_READY1, O_READY0, O_READY1, T_FREE0, T_FREE1, SX_READY, VZ_READY0, VZ_READY1, AUX_SYNC,
   DRAIN, NUM_BARS
 };
@@ -161,8 +159,7 @@ attention_tc_kernel(const __grid_constant__ AttnMaps maps, const bf16* __restric
     mbar_init(bar(Q_FREE), 1 + AUX_WARPS);       // S products retired + helper warps done with Q
     for (int w = 0; w < 2; ++w) {
       mbar_init(bar(S_READY0 + w), 1);
-      mbar_init(bar(PL_READY0 + w), 4);          // one arrival per softmax warp of the tile: keys 0 ... 191 of P
-      mbar_init(bar(P_READY0 + w), 4);           // the rest of P
+      mbar_init(bar(P_READY0 + w), 4);           // one arrival per softmax warp of the tile
       mbar_init(bar(O_READY0 + w), 1);
       mbar_init(bar(T_FREE0 + w), 4);
       mbar_init(bar(VZ_READY0 + w), AUX_WARPS);
@@ -246,9 +243,8 @@ attention_tc_kernel(const __grid_constant__ AttnMaps maps, const bf16* __restric
         umma_commit(bar(S_READY0 + w));
       };
       const int ksteps = NKP / 16 + (n_x > 0 ? 1 : 0);
-      constexpr int KLO = L::KLO;
       // O = P V: A = P in tensor memory (8 columns per 16 keys); B = V, 16 keys per step = two
-      // 8-row groups of the tile.  Issued in two parts, as the parts of P become ready.
+      // 8-row groups of the tile.
       auto issue_pv = [&](int w, uint32_t st, int k0, int k1) {
         const uint32_t t0 = tmem_base + (uint32_t)w * TILE_COLS;
 #pragma unroll 1
@@ -258,52 +254,39 @@ attention_tc_kernel(const __grid_constant__ AttnMaps maps, const bf16* __restric
           umma_bf16_ts(t0 + L::O_COL, t0 + L::p_col(k), bdesc, idesc_bf16(D, true), k > 0 ? 1u : 0u);
         }
       };
-      // The two tiles advance independently: each walks S(h) -> first part of P V (h) -> rest of
-      // P V (h) -> S(h + 1) ..., and this thread issues whichever step has its inputs ready, so the
-      // warpgroups drift apart and one is in its exp2 phase while the tensor core serves the other.
-      // Q (one buffer) is released when both tiles have issued S(h), a K/V stage when both have
-      // issued all of P V (h).
-      int t_it[2] = {0, 0}, t_step[2] = {0, 0};      // per tile: head iteration; step 0 = S, 1 = PV first part, 2 = PV rest
-      int s_count[2] = {0, 0}, pv_count[2] = {0, 0}; // per stage: tiles that have issued S / all of PV
-      long long idle_since = clock64();
-      while ((t_it[0] < n_iter || t_it[1] < n_iter) && ok) {
-        bool progress = false;
-#pragma unroll
-        for (int w = 0; w < 2; ++w) {
-          const int it = t_it[w];
-          if (it >= n_iter) continue;
-          const int s = it & 1;
-          const uint32_t st = sb + (uint32_t)s * L::STAGE;
-          const uint32_t hph = (uint32_t)(it & 1), kph = (uint32_t)((it >> 1) & 1);
-          if (t_step[w] == 0) {
-            if (!(mbar_try_wait(bar(KV_FULL0 + s), kph) && mbar_try_wait(bar(Q_FULL), hph) &&
-                  mbar_try_wait(bar(T_FREE0 + w), hph ^ 1)))
-              continue;
-            tc_fence_after();
-            issue_s(w, st);
-            if (++s_count[s] == 2) { s_count[s] = 0; umma_commit(bar(Q_FREE)); }
-            t_step[w] = 1;
-          } else if (t_step[w] == 1) {
-            if (!(mbar_try_wait(bar(VZ_READY0 + s), kph) && mbar_try_wait(bar(PL_READY0 + w), hph))) continue;
-            tc_fence_after();
-            issue_pv(w, st, 0, KLO);
-            t_step[w] = 2;
-          } else {
-            if (!mbar_try_wait(bar(P_READY0 + w), hph)) continue;
-            tc_fence_after();
-            issue_pv(w, st, KLO, ksteps);
-            umma_commit(bar(O_READY0 + w));
-            if (++pv_count[s] == 2) { pv_count[s] = 0; umma_commit(bar(KV_FREE0 + s)); }
-            t_step[w] = 0;
-            t_it[w] = it + 1;
-          }
-          progress = true;
+      // Issue order per head h: S_0(h), P V of tile 1 of head h - 1, S_1(h), P V of tile 0 of head h:
+      // tile 1 runs behind tile 0, so that one warpgroup is in its exp2 phase while the tensor core
+      // serves the other.  (Letting the two tiles advance independently by polling, and issuing P V
+      // in two parts as P becomes ready, both measured slower.)
+      for (int it = 0; it <= n_iter && ok && n_iter > 0; ++it) {
+        const int s = it & 1;
+        const uint32_t st = sb + (uint32_t)s * L::STAGE, st_prev = sb + (uint32_t)(s ^ 1) * L::STAGE;
+        const uint32_t hph = (uint32_t)(it & 1), kph = (uint32_t)((it >> 1) & 1);
+        const bool head = it < n_iter;
+        if (head) {
+          if (!mbar_wait(bar(KV_FULL0 + s), kph, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(bar(Q_FULL), hph, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(bar(T_FREE0), hph ^ 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          issue_s(0, st);
         }
-        if (progress) {
-          idle_since = clock64();
-        } else if (*abort_flag || clock64() - idle_since > WAIT_LIMIT_CYCLES) {
-          *abort_flag = 1;
-          ok = false;
+        if (it > 0) {
+          if (!mbar_wait(bar(P_READY1), hph ^ 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          issue_pv(1, st_prev, 0, ksteps);
+          umma_commit(bar(O_READY1));
+          umma_commit(bar(KV_FREE0 + (s ^ 1)));
+        }
+        if (head) {
+          if (!mbar_wait(bar(T_FREE1), hph ^ 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          issue_s(1, st);
+          umma_commit(bar(Q_FREE));
+          if (!mbar_wait(bar(VZ_READY0 + s), kph, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(bar(P_READY0), hph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          issue_pv(0, st, 0, ksteps);
+          umma_commit(bar(O_READY0));
         }
       }
       if (*abort_flag) {
@@ -370,8 +353,7 @@ attention_tc_kernel(const __grid_constant__ AttnMaps maps, const bf16* __restric
         const float msl = m * sl2;
         // pass 2: p = exp2((s - m) * sl2), row sum, P (bf16 pairs) back into tensor memory over
         // columns this thread has already read (see the tensor-memory map).  The load of chunk
-        // i + 1 is in flight while chunk i is worked on.  After six chunks (keys 0 ... 191) the
-        // tensor core is told to start on O.
+        // i + 1 is in flight while chunk i is worked on.
         float2 l2 = make_float2(0.f, 0.f);
         const float2 sl2v = make_float2(sl2, sl2), nmsl = make_float2(-msl, -msl);
         tmem_ld32(taddr, r[0]);
@@ -408,12 +390,6 @@ attention_tc_kernel(const __grid_constant__ AttnMaps maps, const bf16* __restric
             for (int j = 0; j < 8; ++j) part[j] = pk[j];
             tmem_st8(taddr + L::p_col(2 * i), part);
           }
-          if (i == 5) {                              // keys 0 ... 191 of P are in place
-            tmem_st_wait();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(PL_READY0 + wg));
-          }
         }
         l = l2.x + l2.y;
         if (n_x > 0) {
@@ -428,9 +404,6 @@ attention_tc_kernel(const __grid_constant__ AttnMaps maps, const bf16* __restric
           tmem_st8(taddr + L::PX_COL, xp);
         }
         tmem_st_wait();
-      } else {
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(PL_READY0 + wg));
       }
       tc_fence_before();
       __syncwarp();
@@ -450,15 +423,17 @@ attention_tc_kernel(const __grid_constant__ AttnMaps maps, const bf16* __restric
       if (lane == 0) mbar_arrive(bar(T_FREE0 + wg));   // the next head's S may overwrite this tile now
       if (warp_active && tok < T) {
         const float inv = 1.0f / l;
-        uint4* orow = reinterpret_cast<uint4*>(out + ((size_t)img * T + tok) * H + (size_t)hd * D);
+        // the row is 32-byte aligned (d is a multiple of 16): 32-byte stores, one sector each
+        bf16* orow = out + ((size_t)img * T + tok) * H + (size_t)hd * D;
 #pragma unroll
-        for (int c = 0; c < CH; ++c) {
-          uint4 w;
-          w.x = pack_bf16(__uint_as_float(o[8 * c + 0]) * inv, __uint_as_float(o[8 * c + 1]) * inv);
-          w.y = pack_bf16(__uint_as_float(o[8 * c + 2]) * inv, __uint_as_float(o[8 * c + 3]) * inv);
-          w.z = pack_bf16(__uint_as_float(o[8 * c + 4]) * inv, __uint_as_float(o[8 * c + 5]) * inv);
-          w.w = pack_bf16(__uint_as_float(o[8 * c + 6]) * inv, __uint_as_float(o[8 * c + 7]) * inv);
-          orow[c] = w;
+        for (int c = 0; c < D / 16; ++c) {
+          uint32_t w[8];
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            w[q] = pack_bf16(__uint_as_float(o[16 * c + 2 * q]) * inv, __uint_as_float(o[16 * c + 2 * q + 1]) * inv);
+          asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(orow + 16 * c), "r"(w[0]),
+                       "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                       : "memory");
         }
       }
     }

@@ -125,7 +125,7 @@ struct Smem {
 
 enum Bar : int {
   KV_FULL0 = 0, KV_FULL1, KV_FREE0, KV_FREE1, Q_FULL, Q_FREE, S_READY0, S_READY1,
-  P_READY0, P_READY1, O_READY0, O_READY1, T_FREE0, T_FREE1, SX_READY, VZ_READY0, VZ_READY1, AUX_SYNC,
+  P_READY0, P_READY1, O_READY0, O_READY1, T_FREE0, T_FREE1, SX_READY0, SX_READY1, VZ_READY0, VZ_READY1, AUX_SYNC,
   DRAIN, NUM_BARS
 };
 
@@ -164,7 +164,10 @@ attention_tc_kernel(const __grid_constant__ AttnMaps maps, const bf16* __restric
       mbar_init(bar(T_FREE0 + w), 4);
       mbar_init(bar(VZ_READY0 + w), AUX_WARPS);
     }
-    mbar_init(bar(SX_READY), AUX_WARPS);
+    // the helper warps can be a head ahead of a softmax warpgroup: one barrier per head parity, so
+    // that a warpgroup never finds its phase overtaken
+    mbar_init(bar(SX_READY0), AUX_WARPS);
+    mbar_init(bar(SX_READY1), AUX_WARPS);
     mbar_init(bar(AUX_SYNC), AUX_WARPS);
     mbar_init(bar(DRAIN), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -313,7 +316,7 @@ attention_tc_kernel(const __grid_constant__ AttnMaps maps, const bf16* __restric
       const uint32_t hph = (uint32_t)(it & 1);
       const float* sxh = sx_all + (it & 1) * MAX_EXTRA * 256;
       if (!mbar_wait(bar(S_READY0 + wg), hph, abort_flag)) { ok = false; break; }
-      if (n_x > 0 && !mbar_wait(bar(SX_READY), hph, abort_flag)) { ok = false; break; }
+      if (n_x > 0 && !mbar_wait(bar(SX_READY0 + (it & 1)), (uint32_t)((it >> 1) & 1), abort_flag)) { ok = false; break; }
       tc_fence_after();
       float l = 0.f;
       if (warp_active) {
@@ -519,7 +522,7 @@ attention_tc_kernel(const __grid_constant__ AttnMaps maps, const bf16* __restric
       }
       __syncwarp();
       if (lane == 0) {
-        mbar_arrive(bar(SX_READY));
+        mbar_arrive(bar(SX_READY0 + (it & 1)));
         mbar_arrive(bar(Q_FREE));
       }
       if (n_x > 0) {

@@ -172,8 +172,11 @@ def test_attention_bf16(ctx, images, T, heads, d, spread):
     want = _oracle_attention(qr, images, T, heads)
     got = out.float().cpu().numpy()
     assert np.isfinite(got).all()
-    # P is rounded to bf16 before PV and the output is bf16: errors of a few bf16 ulps of |V|max
-    assert np.abs(got - want).max() <= 3 * BF16_EPS * np.abs(qr[:, 2 * H:]).max()
+    # P is rounded to bf16 before PV and the output is bf16.  With near-uniform attention the
+    # rounding errors of P average out, so the bound scales with the outputs, not with |V|max:
+    # two bf16 half-ulps of the largest output plus a small share of |V|max.
+    vmax = np.abs(qr[:, 2 * H:]).max()
+    assert np.abs(got - want).max() <= 2 * BF16_EPS * np.abs(want).max() + 5e-4 * vmax
 
 
 def test_attention_bf16_identical_keys_gives_mean_of_values(ctx):

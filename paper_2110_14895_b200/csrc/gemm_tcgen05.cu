@@ -66,18 +66,29 @@ template <int BN, int CTAS> __host__ __device__ constexpr uint32_t make_idesc() 
 
 // gelu(v) = 0.5 v (1 + erf(v / sqrt 2)) = max(v, 0) - 0.5 |v| erfc(|v| / sqrt 2), with
 // erfc(z) = (a1 t + ... + a5 t^5) exp(-z^2), t = 1 / (1 + p z), z >= 0 (Abramowitz & Stegun
-// 7.1.26, |error| <= 1.5e-7), on the MUFU reciprocal and exp2.  The factor 0.5 is folded into
-// the coefficients and 1/sqrt 2 into p and the exponent scale.
-__device__ __forceinline__ float gelu_erf(float v) {
-  const float a = fabsf(v);
-  float t, e;
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.3275911f * 0.70710678118654752440f, a, 1.0f)));
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(a * a * (-0.5f * 1.4426950408889634f)));
-  float q = fmaf(0.5f * 1.061405429f, t, 0.5f * -1.453152027f);
-  q = fmaf(q, t, 0.5f * 1.421413741f);
-  q = fmaf(q, t, 0.5f * -0.284496736f);
-  q = fmaf(q, t, 0.5f * 0.254829592f);
-  return fmaxf(v, 0.f) - q * t * e * a;
+// 7.1.26, |error| <= 1.5e-7), on the MUFU reciprocal and exp2.  The factor -0.5 is folded into
+// the coefficients and 1/sqrt 2 into p and the exponent scale.  Two values per call: the
+// polynomial and the products run as packed two-wide fp32 instructions (9 instructions and
+// 2 MUFU operations per value).
+__device__ __forceinline__ float2 gelu_erf2(float2 v) {
+  const float2 a = make_float2(fabsf(v.x), fabsf(v.y));
+  const float kp = 0.3275911f * 0.70710678118654752440f;
+  const float2 den = __ffma2_rn(make_float2(kp, kp), a, make_float2(1.0f, 1.0f));
+  float2 t, e;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t.x) : "f"(den.x));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t.y) : "f"(den.y));
+  const float ke = -0.5f * 1.4426950408889634f;
+  const float2 arg = __fmul2_rn(__fmul2_rn(a, a), make_float2(ke, ke));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.x) : "f"(arg.x));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.y) : "f"(arg.y));
+  const float c5 = -0.5f * 1.061405429f, c4 = -0.5f * -1.453152027f, c3 = -0.5f * 1.421413741f,
+              c2 = -0.5f * -0.284496736f, c1 = -0.5f * 0.254829592f;
+  float2 q = __ffma2_rn(make_float2(c5, c5), t, make_float2(c4, c4));
+  q = __ffma2_rn(q, t, make_float2(c3, c3));
+  q = __ffma2_rn(q, t, make_float2(c2, c2));
+  q = __ffma2_rn(q, t, make_float2(c1, c1));
+  const float2 r = make_float2(fmaxf(v.x, 0.f), fmaxf(v.y, 0.f));
+  return __ffma2_rn(__fmul2_rn(q, a), __fmul2_rn(t, e), r);
 }
 
 struct TcParams {
@@ -314,7 +325,11 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
           }
           if (EPI == EPI_BIAS_GELU) {
 #pragma unroll
-            for (int e = 0; e < 64; ++e) v[e] = gelu_erf(v[e]);
+            for (int e = 0; e < 64; e += 2) {
+              const float2 y = gelu_erf2(make_float2(v[e], v[e + 1]));
+              v[e] = y.x;
+              v[e + 1] = y.y;
+            }
           }
           if (EPI == EPI_BIAS_RESIDUAL) {
             if (!mbar_wait(rb, rphase, abort_flag)) { ok = false; break; }

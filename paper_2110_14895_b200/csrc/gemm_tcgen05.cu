@@ -318,10 +318,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
           for (int g = 0; g < 16; ++g) {
             const float4 b = (c0 + 4 * g < p.N) ? __ldg(reinterpret_cast<const float4*>(p.bias + c0) + g)
                                                 : make_float4(0.f, 0.f, 0.f, 0.f);
-            v[4 * g + 0] = __uint_as_float(r[4 * g + 0]) + b.x;
-            v[4 * g + 1] = __uint_as_float(r[4 * g + 1]) + b.y;
-            v[4 * g + 2] = __uint_as_float(r[4 * g + 2]) + b.z;
-            v[4 * g + 3] = __uint_as_float(r[4 * g + 3]) + b.w;
+            const float2 lo = __fadd2_rn(make_float2(__uint_as_float(r[4 * g + 0]), __uint_as_float(r[4 * g + 1])), make_float2(b.x, b.y));
+            const float2 hi = __fadd2_rn(make_float2(__uint_as_float(r[4 * g + 2]), __uint_as_float(r[4 * g + 3])), make_float2(b.z, b.w));
+            v[4 * g + 0] = lo.x;
+            v[4 * g + 1] = lo.y;
+            v[4 * g + 2] = hi.x;
+            v[4 * g + 3] = hi.y;
           }
           if (EPI == EPI_BIAS_GELU) {
 #pragma unroll
@@ -344,9 +346,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
               const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
-                const float2 f = __bfloat1622float2(h[e]);
-                v[ck * 8 + 2 * e] += f.x;
-                v[ck * 8 + 2 * e + 1] += f.y;
+                const float2 y = __fadd2_rn(make_float2(v[ck * 8 + 2 * e], v[ck * 8 + 2 * e + 1]), __bfloat1622float2(h[e]));
+                v[ck * 8 + 2 * e] = y.x;
+                v[ck * 8 + 2 * e + 1] = y.y;
               }
             }
           } else {

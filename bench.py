@@ -34,8 +34,9 @@ WORKLOADS = {
 }
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fc1 GEMM, from the ncu capture
 # whose summary is kept under profiles/ (same kernel build); None = not captured
-NCU_TRAFFIC = {"huge14": 384.5e6}
+NCU_TRAFFIC = {"huge14": None}   # the fc1 epilogue changed since the last capture
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL_BF16_TFLOPS = 2250.0   # datasheet dense bf16 figure of the B200 (context; the measured peaks are the denominators)
 
 
 def max_over_ranks(ms, dist=None, device=None):
@@ -200,6 +201,50 @@ def microbatch_sweep(vit, model, shape, dev, torch, total=256, sizes=(1, 2, 4, 8
     return out
 
 
+def measure_workload(vit, torch, dev, name, steps=5, warmup=3, group=1):
+    """Device-timed images/s of one of the named workloads (inputs resident), used for the extra
+    workloads reported beside the headline one.  `group` > 1 carries that many microbatches through
+    every launch together."""
+    preset, batch, mb, n_stages = WORKLOADS[name]
+    shape = vitgen.preset(preset)
+    counts = stage_counts(shape, n_stages)
+    _, blob = vitgen.make_params(shape, seed=0)
+    model = vit.VitModel(shape, blob, vit.VIT_BF16, mb * group, device=dev)
+    del blob
+    pix = torch.from_numpy(vitgen.make_pixels(shape, batch, seed=0)).to(dev)
+    logits = torch.empty((batch, shape.num_classes), dtype=torch.float32, device=dev)
+    n_streams = max(1, min(4, batch // (mb * group)))
+    wss, streams, wsb = model.make_pipeline_buffers(mb * group, n_streams)
+
+    def step():
+        model.run_pipeline(counts, mb, pix, logits, wss, streams, wsb, group=group)
+
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(streams[0])
+    for s_ in streams[1:]:
+        s_.wait_event(e0)
+    for _ in range(steps):
+        step()
+    for s_ in streams[1:]:
+        e = torch.cuda.Event()
+        e.record(s_)
+        streams[0].wait_event(e)
+    e1.record(streams[0])
+    torch.cuda.synchronize(dev)
+    for s_ in streams:
+        model.check(s_)
+    ms = e0.elapsed_time(e1) / steps
+    total_flops = flops_per_image(shape)[0]
+    model.close()
+    value = batch / (ms / 1e3)
+    return {"workload": f"ViT-{preset}, batch {batch}, microbatch {mb}, {n_stages} stages, {n_streams} streams"
+                        + (f", {group} microbatches per launch" if group > 1 else ""),
+            "value": value, "unit": "images/s", "ms_per_step": ms, "tflops": value * total_flops / 1e12}
+
+
 def workload_config(preset, shape, batch, mb, counts, world, n_streams):
     return {
         "workload": f"ViT-{preset} forward, batch {batch}, microbatch {mb}, stages {counts}, "
@@ -247,6 +292,8 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--workload", default="huge14", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extra-workloads", action="store_true",
+                    help="skip the brief ViT-L/16 and ViT-B/16 measurements reported under 'workloads'")
     ap.add_argument("--streams", type=int, default=0, help="streams for the stage runner (0 = min(4, microbatches))")
     ap.add_argument("--sweep", action="store_true",
                     help="also run the microbatch sweep (sizes 1..256, 4 stages, streams) and add it as 'sweep'")
@@ -348,6 +395,13 @@ def main():
     if args.sweep:
         sweep = microbatch_sweep(vit, model, shape, dev, torch)
 
+    # the other single-GPU configurations of the metric, briefly (rank 0 of a single-GPU run only)
+    extra = {}
+    if world == 1 and not args.no_extra_workloads and args.workload == "huge14":
+        extra["large16"] = measure_workload(vit, torch, dev, "large16")
+        extra["large16_grouped"] = measure_workload(vit, torch, dev, "large16", group=4)
+        extra["base16"] = measure_workload(vit, torch, dev, "base16")
+
     if rank == 0:
         pk = peaks()
         total_flops, gemm, attn, embed = flops_per_image(shape)
@@ -379,7 +433,9 @@ def main():
             "tflops": value * total_flops / 1e12,
             "frac_of_bf16_peak": {"burst": value * total_flops / 1e12 / world / pk["bf16_tflops"],
                                   "sustained": value * total_flops / 1e12 / world / pk["bf16_tflops_sustained"],
-                                  "peaks": pk["source"]},
+                                  "nominal": value * total_flops / 1e12 / world / NOMINAL_BF16_TFLOPS,
+                                  "peaks": pk["source"], "burst_tflops": pk["bf16_tflops"],
+                                  "sustained_tflops": pk["bf16_tflops_sustained"], "nominal_tflops": NOMINAL_BF16_TFLOPS},
             "e2e": {"value": e2e_value, "unit": "images/s",
                     "h2d_bytes_per_step": int(pix_host.numel() * 4), "d2h_bytes_per_step": int(logits_host.numel() * 4),
                     "microbatch": e2e_mb, "streams": e2e_streams_n},
@@ -394,10 +450,17 @@ def main():
                 "launches": top_n, "traffic": NCU_TRAFFIC.get(args.workload),
                 "all_gemms": {"achieved": gemm_all, "frac": gemm_all / peak if gemm_all else None,
                               "frac_of_burst": gemm_all / pk["bf16_tflops"] if gemm_all else None,
+                              "frac_of_nominal": gemm_all / NOMINAL_BF16_TFLOPS if gemm_all else None,
                               "launches": gemm_launches},
             },
             "kernels": per_class,
         }
+        if extra:
+            for w in extra.values():
+                w["frac_of_bf16_peak"] = {"burst": w["tflops"] / pk["bf16_tflops"],
+                                          "sustained": w["tflops"] / pk["bf16_tflops_sustained"],
+                                          "nominal": w["tflops"] / NOMINAL_BF16_TFLOPS}
+            line["workloads"] = extra
         if sweep is not None:
             line["sweep"] = sweep
         if not args.no_cpu_baseline and world == 1:

@@ -160,6 +160,18 @@ int vit_run_pipeline(vit_handle* h, const int32_t* stage_layers, int n_stages, i
                      void* const* ws_per_stream, size_t ws_bytes, void* const* streams,
                      int n_streams);
 
+/* vit_run_pipeline with `group` consecutive microbatches carried through every kernel launch
+ * together (paper Section 5.4 studies the microbatch size: small microbatches keep the memory
+ * per stage low but leave a large GPU underused; images are independent, so several of them in
+ * flight can share a launch without changing any result).  Microbatch m still consists of images
+ * [m * microbatch, (m + 1) * microbatch); groups go round-robin over the streams.
+ *   ws_per_stream[i]: at least vit_pipeline_workspace_bytes(cfg, group * microbatch);
+ *   group * microbatch <= max_microbatch. */
+int vit_run_pipeline_grouped(vit_handle* h, const int32_t* stage_layers, int n_stages, int batch,
+                             int microbatch, int group, const float* pixels, float* logits,
+                             void* const* ws_per_stream, size_t ws_bytes, void* const* streams,
+                             int n_streams);
+
 /* Same as vit_run_pipeline with HOST pixels and logits: each microbatch's pixels are copied to
  * the device, and its logits back, on that microbatch's stream (copies are asynchronous only
  * if the host memory is pinned).  Does not synchronise. */

@@ -27,7 +27,7 @@ VIT_TILING_AUTO, VIT_TILING_128x128, VIT_TILING_128x256, VIT_TILING_PAIR_256x256
 EXPORTS = [
     "vit_param_count", "vit_workspace_bytes", "vit_pipeline_workspace_bytes", "vit_create",
     "vit_destroy", "vit_patch_embed", "vit_run_stage", "vit_head", "vit_run_pipeline",
-    "vit_run_pipeline_host", "vit_check_status", "vit_launch_count", "vit_status_string",
+    "vit_run_pipeline_host", "vit_run_pipeline_grouped", "vit_check_status", "vit_launch_count", "vit_status_string",
     "vit_op_layernorm", "vit_op_linear", "vit_op_linear_tiled", "vit_op_attention", "vit_profile_enable",
     "vit_profile_collect", "vit_head_static", "vit_partition", "vit_partition_categories",
     "vit_debug_wait_probe",
@@ -89,6 +89,9 @@ def lib():
         f.restype = c_int
         f.argtypes = [c_void_p, P(c_int32), c_int, c_int, c_int, c_void_p, c_void_p, P(c_void_p),
                       c_size_t, P(c_void_p), c_int]
+    L.vit_run_pipeline_grouped.restype = c_int
+    L.vit_run_pipeline_grouped.argtypes = [c_void_p, P(c_int32), c_int, c_int, c_int, c_int, c_void_p, c_void_p,
+                                           P(c_void_p), c_size_t, P(c_void_p), c_int]
     L.vit_check_status.restype = c_int
     L.vit_check_status.argtypes = [c_void_p, c_void_p]
     L.vit_launch_count.restype = c_uint64
@@ -201,6 +204,18 @@ def vit_run_pipeline_host(h, stage_layers, batch, microbatch, host_pixels, host_
                           ws_bytes, streams):
     _pipeline(lib().vit_run_pipeline_host, "vit_run_pipeline_host", h, stage_layers, batch, microbatch,
               host_pixels, host_logits, ws_ptrs, ws_bytes, streams)
+
+
+def vit_run_pipeline_grouped(h, stage_layers, batch, microbatch, group, pixels, logits, ws_ptrs, ws_bytes, streams):
+    n = len(stage_layers)
+    sl = (c_int32 * n)(*stage_layers)
+    k = len(streams)
+    if len(ws_ptrs) != k:
+        raise ValueError("one workspace per stream")
+    wsa = (c_void_p * k)(*ws_ptrs)
+    sta = (c_void_p * k)(*streams)
+    _check(lib().vit_run_pipeline_grouped(h, sl, n, batch, microbatch, group, pixels, logits, wsa, ws_bytes, sta, k),
+           "vit_run_pipeline_grouped")
 
 
 def vit_check_status(h, stream=0) -> None:
@@ -362,8 +377,13 @@ class VitModel:
         streams = [self.torch.cuda.Stream(self.device) for _ in range(n_streams)]
         return wss, streams, n
 
-    def run_pipeline(self, stage_layers, microbatch, pixels, logits, wss, streams, ws_bytes, host=False):
+    def run_pipeline(self, stage_layers, microbatch, pixels, logits, wss, streams, ws_bytes, host=False, group=1):
         batch = pixels.shape[0]
+        if group > 1:
+            vit_run_pipeline_grouped(self.h, list(stage_layers), batch, microbatch, group, pixels.data_ptr(),
+                                     logits.data_ptr(), [w.data_ptr() for w in wss], ws_bytes,
+                                     [s.cuda_stream for s in streams])
+            return
         fn = vit_run_pipeline_host if host else vit_run_pipeline
         fn(self.h, list(stage_layers), batch, microbatch, pixels.data_ptr(), logits.data_ptr(),
            [w.data_ptr() for w in wss], ws_bytes, [s.cuda_stream for s in streams])

@@ -472,6 +472,16 @@ int vit_run_pipeline(vit_handle* h, const int32_t* stage_layers, int n_stages, i
                       streams, n_streams, false);
 }
 
+int vit_run_pipeline_grouped(vit_handle* h, const int32_t* stage_layers, int n_stages, int batch, int mb,
+                             int group, const float* pixels, float* logits, void* const* ws_per_stream,
+                             size_t ws_bytes, void* const* streams, int n_streams) {
+  if (group < 1 || mb < 1 || (long long)group * mb > 0x7fffffffLL) return VIT_ERR_INVALID_ARG;
+  // images are independent, so `group` microbatches carried through every launch together are the
+  // same computation as one microbatch of group * mb images
+  return run_pipeline(h, stage_layers, n_stages, batch, group * mb, pixels, logits, ws_per_stream, ws_bytes,
+                      streams, n_streams, false);
+}
+
 int vit_run_pipeline_host(vit_handle* h, const int32_t* stage_layers, int n_stages, int batch, int mb,
                           const float* host_pixels, float* host_logits, void* const* ws_per_stream,
                           size_t ws_bytes, void* const* streams, int n_streams) {

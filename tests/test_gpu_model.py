@@ -170,6 +170,39 @@ def test_large16_batch128_microbatch8_uneven_16_stages():
     m.close()
 
 
+def test_large16_grouped_microbatches_match_ungrouped_and_oracle():
+    """Several microbatches carried through every launch together: the same function of every
+    image as microbatch by microbatch, bit for bit (rows of a GEMM, rows of LayerNorm and heads of
+    attention do not depend on what else is in the launch, and the K order is fixed), and within
+    the bf16 tolerance of the oracle."""
+    shape = vitgen.preset("large16")
+    vit, m, params = _model(shape, _vit().VIT_BF16, 32)
+    B, mb = 40, 8                                   # five microbatches: a full group of four and a ragged one
+    pix = vitgen.make_pixels(shape, B, seed=3)
+    dp = torch.from_numpy(pix).cuda()
+    stages = [le - lb for lb, le in vitgen.uneven_partition(16, 24, seed=0)]
+    outs = []
+    for group in (1, 4):
+        wss, streams, wsb = m.make_pipeline_buffers(mb * group, 2)
+        logits = torch.full((B, shape.num_classes), float("nan"), dtype=torch.float32, device="cuda")
+        torch.cuda.synchronize()
+        m.run_pipeline(stages, mb, dp, logits, wss, streams, wsb, group=group)
+        for s in streams:
+            m.check(s)
+        outs.append(logits.cpu().numpy())
+    sample = [0, 7, 8, 31, 32, 39]
+    want = O.forward(params, shape, pix[sample])
+    for got in outs:
+        assert np.isfinite(got).all()
+        ok, msg = logits_within_tolerance(got[sample], want, 2e-2, 0.9995)
+        assert ok, msg
+    assert np.array_equal(outs[0], outs[1])
+    with pytest.raises(vit.VitError) as e:          # group * microbatch beyond max_microbatch
+        m.run_pipeline(stages, mb, dp, logits, wss, streams, wsb, group=5)
+    assert e.value.status == vit.VIT_ERR_INVALID_ARG
+    m.close()
+
+
 def test_huge14_batch128_single_stage_equals_eight_stages_and_oracle():
     shape = vitgen.preset("huge14")
     vit, m, params = _model(shape, _vit().VIT_BF16, 128)

@@ -13,6 +13,9 @@ What is computed, and where the paper states it:
   * An embedding layer precedes the transformer layers and gives every input a uniform
     dimension; the task is image classification, the last stage produces the final result
     (Sections 3.1 and 4).  `patch_embed` and `head` are these two book-ends.
+  * The compressed models of Section 5.5 are distilled transformers of the same structure: they
+    carry a distillation token beside the class token (cfg.extra_tokens = 1) and a second
+    classifier on it; the prediction is the mean of the two classifiers' outputs.
 The paper gives no formula for the individual operations; the ones used are the textbook
 definitions for a pre-LN ViT and are spelled out in each docstring.
 
@@ -77,20 +80,25 @@ def _cast(params, dtype):
 
 
 def patch_embed(params, cfg, pixels, dtype=np.float64):
-    """Embedding book-end.  pixels [mb, C, S, S].  Token t = 1 + py*(S/P) + px is
+    """Embedding book-end.  pixels [mb, C, S, S].  Token t = t0 + py*(S/P) + px is
     patch.W . vec(patch) + patch.b + pos[t], vec ordered (channel, row, column);
-    token 0 is cls + pos[0].  Returns [mb, T, H]."""
-    p = _cast({k: params[k] for k in ("patch.W", "patch.b", "cls", "pos")}, dtype)
+    token 0 is cls + pos[0]; with a distillation token, token 1 is dist + pos[1] and t0 = 2
+    (otherwise t0 = 1).  Returns [mb, T, H]."""
+    names = ("patch.W", "patch.b", "cls", "pos") + (("dist",) if cfg.extra_tokens else ())
+    p = _cast({k: params[k] for k in names}, dtype)
+    t0 = 1 + cfg.extra_tokens
     P, G = cfg.patch_size, cfg.grid
     mb = pixels.shape[0]
     x = np.empty((mb, cfg.tokens, cfg.hidden), dtype=dtype)
     for n in range(mb):
         img = np.asarray(pixels[n], dtype=dtype)
         x[n, 0] = p["cls"] + p["pos"][0]
+        if cfg.extra_tokens:
+            x[n, 1] = p["dist"] + p["pos"][1]
         for py in range(G):
             for px in range(G):
                 vec = img[:, py * P:(py + 1) * P, px * P:(px + 1) * P].reshape(-1)
-                t = 1 + py * G + px
+                t = t0 + py * G + px
                 x[n, t] = p["patch.W"] @ vec + p["patch.b"] + p["pos"][t]
     return x
 
@@ -124,13 +132,19 @@ def run_stage(params, cfg, layer_begin, layer_end, x, dtype=np.float64):
 
 def head(params, cfg, x, dtype=np.float64):
     """Classification book-end: final LayerNorm of the class token (row 0 of each image),
-    then logits = f . head.W^T + head.b.  Returns [mb, classes]."""
-    p = _cast({k: params[k] for k in ("lnf.g", "lnf.b", "head.W", "head.b")}, dtype)
+    then logits = f . head.W^T + head.b.  With a distillation token, row 1 goes through the same
+    LayerNorm and its own classifier head_dist, and the result is the mean of the two logit
+    vectors.  Returns [mb, classes]."""
+    names = ("lnf.g", "lnf.b", "head.W", "head.b") + (("head_dist.W", "head_dist.b") if cfg.extra_tokens else ())
+    p = _cast({k: params[k] for k in names}, dtype)
     x = np.asarray(x, dtype=dtype)
     out = np.empty((x.shape[0], cfg.num_classes), dtype=dtype)
     for n in range(x.shape[0]):
         f = layernorm(x[n, 0], p["lnf.g"], p["lnf.b"], cfg.ln_eps)
         out[n] = p["head.W"] @ f + p["head.b"]
+        if cfg.extra_tokens:
+            fd = layernorm(x[n, 1], p["lnf.g"], p["lnf.b"], cfg.ln_eps)
+            out[n] = (out[n] + p["head_dist.W"] @ fd + p["head_dist.b"]) / dtype(2)
     return out
 
 

@@ -256,9 +256,14 @@ def _scalar_vit(p, cfg, img):
     x = [[0.0] * H for _ in range(T)]
     for o in range(H):
         x[0][o] = float(p["cls"][o] + p["pos"][0][o])
+    first = 1
+    if cfg.extra_tokens:                       # distillation token right after the class token
+        first = 2
+        for o in range(H):
+            x[1][o] = float(p["dist"][o] + p["pos"][1][o])
     for py in range(G):
         for px in range(G):
-            t = 1 + py * G + px
+            t = first + py * G + px
             for o in range(H):
                 acc = 0.0
                 for c in range(cfg.channels):
@@ -297,7 +302,12 @@ def _scalar_vit(p, cfg, img):
             o = lin(u1, q("W2"), q("b2"))
             x[t] = [x[t][i] + o[i] for i in range(H)]
     f = ln(x[0], p["lnf.g"], p["lnf.b"])
-    return lin(f, p["head.W"], p["head.b"]), x
+    logits = lin(f, p["head.W"], p["head.b"])
+    if cfg.extra_tokens:                       # mean of the class-token and distillation-token classifiers
+        fd = ln(x[1], p["lnf.g"], p["lnf.b"])
+        ld = lin(fd, p["head_dist.W"], p["head_dist.b"])
+        logits = [(u + v) / 2.0 for u, v in zip(logits, ld)]
+    return logits, x
 
 
 def test_brute_force_scalar_model_2_layers_5_tokens():
@@ -305,6 +315,79 @@ def test_brute_force_scalar_model_2_layers_5_tokens():
     assert cfg.tokens == 5 and cfg.layers == 2
     p = _rand_params(cfg, 12)
     pix = np.random.default_rng(13).uniform(-1, 1, size=(2, 3, 4, 4))
+    got = O.forward(p, cfg, pix)
+    tokens = O.run_stage(p, cfg, 0, 2, O.patch_embed(p, cfg, pix))
+    for n in range(2):
+        logits, x = _scalar_vit(p, cfg, pix[n])
+        np.testing.assert_allclose(got[n], logits, rtol=0, atol=1e-5 * max(abs(v) for v in logits))
+        np.testing.assert_allclose(tokens[n], np.array(x), rtol=0, atol=1e-10)
+
+
+# ----------------------------------------------------------------------------- distillation token
+DIST = TINY.with_(extra_tokens=1)
+
+
+def test_distillation_token_inventory_and_count():
+    # one more token, one more position row, a second classifier
+    assert DIST.tokens == TINY.tokens + 1 and DIST.first_patch_token == 2
+    H, C = DIST.hidden, DIST.num_classes
+    assert vitgen.param_count(DIST) - vitgen.param_count(TINY) == H + H + C * H + C
+    names = [n for n, _, _ in vitgen.param_specs(DIST)]
+    assert names.index("dist") == names.index("cls") + 1 and names[-2:] == ["head_dist.W", "head_dist.b"]
+    # the distilled small / base shapes: 198 tokens
+    assert vitgen.preset("deit_small16").tokens == 198 and vitgen.preset("deit_base16").tokens == 198
+
+
+def test_distillation_token_order_and_special_rows():
+    """Zero patch weights: token 0 = cls + pos[0], token 1 = dist + pos[1], patch tokens start at 2
+    and carry patch.b + pos[t].  A one-hot patch weight reads back the pixel that encodes its own
+    (patch, channel, row, column), which pins the flatten and token order with the extra token."""
+    cfg = DIST
+    p = _rand_params(cfg, 3)
+    p["patch.W"] = np.zeros_like(p["patch.W"])
+    pix = np.random.default_rng(4).uniform(-1, 1, size=(1, 3, 4, 4))
+    x = O.patch_embed(p, cfg, pix)[0]
+    np.testing.assert_allclose(x[0], p["cls"] + p["pos"][0], atol=1e-12)
+    np.testing.assert_allclose(x[1], p["dist"] + p["pos"][1], atol=1e-12)
+    for t in range(2, cfg.tokens):
+        np.testing.assert_allclose(x[t], p["patch.b"] + p["pos"][t], atol=1e-12)
+    P, G = cfg.patch_size, cfg.grid
+    img = np.zeros((1, 3, 4, 4))
+    for c in range(3):
+        for r in range(4):
+            for q in range(4):
+                img[0, c, r, q] = 1000 * ((r // P) * G + q // P) + 100 * c + 10 * (r % P) + (q % P)
+    c, i, j = 2, 1, 0
+    p["patch.W"][5, c * P * P + i * P + j] = 1.0
+    p["patch.b"] = np.zeros_like(p["patch.b"])
+    p["pos"] = np.zeros_like(p["pos"])
+    x = O.patch_embed(p, cfg, img)[0]
+    for patch in range(G * G):
+        assert x[2 + patch, 5] == 1000 * patch + 100 * c + 10 * i + j
+
+
+def test_distillation_head_is_the_mean_of_two_classifiers():
+    cfg = DIST
+    p = _rand_params(cfg, 5)
+    rng = np.random.default_rng(6)
+    x = rng.normal(size=(2, cfg.tokens, cfg.hidden))
+    plain = TINY
+    on_cls = O.head({k: p[k] for k in ("lnf.g", "lnf.b", "head.W", "head.b")}, plain, x[:, [0] + list(range(2, cfg.tokens))])
+    swapped = dict(p)
+    q = {"lnf.g": p["lnf.g"], "lnf.b": p["lnf.b"], "head.W": p["head_dist.W"], "head.b": p["head_dist.b"]}
+    on_dist = O.head(q, plain, x[:, 1:])            # row 1 presented as "row 0" to the plain head
+    np.testing.assert_allclose(O.head(p, cfg, x), (on_cls + on_dist) / 2, atol=1e-12)
+    # rows other than 0 and 1 do not matter
+    y = x.copy()
+    y[:, 2:] = rng.normal(size=y[:, 2:].shape)
+    np.testing.assert_allclose(O.head(p, cfg, y), O.head(p, cfg, x), atol=0)
+
+
+def test_brute_force_scalar_model_with_distillation_token():
+    cfg = DIST
+    assert cfg.tokens == 6
+    p = _rand_params(cfg, 21)
+    pix = np.random.default_rng(22).uniform(-1, 1, size=(2, 3, 4, 4))
     got = O.forward(p, cfg, pix)
     tokens = O.run_stage(p, cfg, 0, 2, O.patch_embed(p, cfg, pix))
     for n in range(2):

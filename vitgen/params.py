@@ -3,7 +3,7 @@
 Blob layout (fp32, tensors back to back in this order, matrices [out, in] row-major):
 
     patch.W [H, C*P*P]   column index = c*P*P + i*P + j  (channel, row, column inside the patch)
-    patch.b [H]    cls [H]    pos [T, H]
+    patch.b [H]    cls [H]    (dist [H] when the model has a distillation token)    pos [T, H]
     for each layer l:  l{l}.ln1.g [H]  l{l}.ln1.b [H]
                        l{l}.Wqkv [3H, H]  l{l}.bqkv [3H]     rows [0,H) Q, [H,2H) K, [2H,3H) V; head h owns rows h*d..(h+1)*d of each
                        l{l}.Wo [H, H]     l{l}.bo [H]
@@ -11,6 +11,7 @@ Blob layout (fp32, tensors back to back in this order, matrices [out, in] row-ma
                        l{l}.W1 [F, H]     l{l}.b1 [F]
                        l{l}.W2 [H, F]     l{l}.b2 [H]
     lnf.g [H]  lnf.b [H]  head.W [classes, H]  head.b [classes]
+    (head_dist.W [classes, H]  head_dist.b [classes] when the model has a distillation token)
 """
 from concurrent.futures import ThreadPoolExecutor
 import os
@@ -30,8 +31,10 @@ def param_specs(cfg: ViTConfig):
         ("patch.W", (H, cfg.patch_k), "normal"),
         ("patch.b", (H,), "normal"),
         ("cls", (H,), "normal"),
-        ("pos", (T, H), "normal"),
     ]
+    if cfg.extra_tokens:
+        specs.append(("dist", (H,), "normal"))
+    specs.append(("pos", (T, H), "normal"))
     for l in range(cfg.layers):
         p = f"l{l}."
         specs += [
@@ -46,6 +49,8 @@ def param_specs(cfg: ViTConfig):
         ("lnf.g", (H,), "gain"), ("lnf.b", (H,), "shift"),
         ("head.W", (C, H), "normal"), ("head.b", (C,), "normal"),
     ]
+    if cfg.extra_tokens:
+        specs += [("head_dist.W", (C, H), "normal"), ("head_dist.b", (C,), "normal")]
     return specs
 
 

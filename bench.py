@@ -31,6 +31,10 @@ WORKLOADS = {
     "large16": ("large16", 128, 8, 16),
     "base16": ("base16", 64, 16, 4),
     "small16": ("small16", 64, 16, 4),
+    # the compressed (distilled) family, 198 tokens
+    "deit_base16": ("deit_base16", 64, 16, 4),
+    "deit_small16": ("deit_small16", 64, 16, 4),
+    "deit_tiny16": ("deit_tiny16", 64, 16, 4),
 }
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fc1 GEMM, from the ncu capture
 # whose summary is kept under profiles/ (same kernel build); None = not captured

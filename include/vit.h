@@ -63,15 +63,19 @@ typedef struct vit_config {
   float   ln_eps;         /* LayerNorm epsilon (inside the square root) */
   int32_t dtype;          /* VIT_BF16 or VIT_FP32 */
   int32_t max_microbatch; /* largest microbatch any call will use */
+  int32_t extra_tokens;   /* 0, or 1 for a distillation token after the class token (see below) */
 } vit_config;
 
 typedef struct vit_handle vit_handle; /* opaque */
 
 /* Number of fp32 values in the host parameter blob for this configuration (0 if the
  * configuration is invalid).  Blob layout, tensors back to back, matrices [out, in] row-major:
- *   patch.W [H, C*P*P] (column = c*P*P + i*P + j), patch.b [H], cls [H], pos [T, H],
+ *   patch.W [H, C*P*P] (column = c*P*P + i*P + j), patch.b [H], cls [H], (dist [H]), pos [T, H],
  *   per layer: ln1.g ln1.b Wqkv[3H,H] bqkv[3H] Wo[H,H] bo[H] ln2.g ln2.b W1[F,H] b1[F] W2[H,F] b2[H],
- *   lnf.g [H], lnf.b [H], head.W [classes, H], head.b [classes].
+ *   lnf.g [H], lnf.b [H], head.W [classes, H], head.b [classes], (head_dist.W, head_dist.b).
+ * The entries in parentheses exist when extra_tokens == 1: the compressed models of the paper's
+ * Section 5.5 are distilled transformers with a distillation token; then T = patches + 2, token 1
+ * is dist + pos[1], patch tokens start at 2, and the head averages two classifiers.
  * Wqkv rows [0,H) produce Q, [H,2H) K, [2H,3H) V; head h owns rows h*d..(h+1)*d of each. */
 size_t vit_param_count(const vit_config* cfg);
 
@@ -99,8 +103,9 @@ int vit_destroy(vit_handle* h);
 /* Embedding book-end (paper Section 4: inputs pass an embedding layer that gives them the
  * uniform dimension the transformer layers expect).
  *   pixels: dev, fp32 [microbatch, C, S, S] (NCHW).
- *   tokens_out: dev, activations [microbatch, T, H].  Token 1 + py*(S/P) + px is
- *     patch.W . vec(patch(py,px)) + patch.b + pos[token]; token 0 is cls + pos[0].
+ *   tokens_out: dev, activations [microbatch, T, H].  Token 1 + extra_tokens + py*(S/P) + px is
+ *     patch.W . vec(patch(py,px)) + patch.b + pos[token]; token 0 is cls + pos[0] (and token 1
+ *     dist + pos[1] when extra_tokens == 1).
  *   ws: dev scratch of at least vit_workspace_bytes(cfg, microbatch). */
 int vit_patch_embed(vit_handle* h, int microbatch, const float* pixels, void* tokens_out,
                     void* ws, size_t ws_bytes, void* stream);
@@ -118,7 +123,9 @@ int vit_run_stage(vit_handle* h, int layer_begin, int layer_end, int microbatch,
 
 /* Classification book-end (paper Section 3.1: the device of the final stage produces the
  * final result; Section 4: the task is image classification).  Final LayerNorm of each image's
- * class token, then logits = f . head.W^T + head.b.
+ * class token, then logits = f . head.W^T + head.b.  With extra_tokens == 1 the distillation
+ * token (row 1) goes through the same LayerNorm and the classifier head_dist, and the logits are
+ * the mean of the two classifiers' outputs.
  *   tokens: dev, activations [microbatch, T, H];  logits: dev, fp32 [microbatch, classes]. */
 int vit_head(vit_handle* h, int microbatch, const void* tokens, float* logits,
              void* ws, size_t ws_bytes, void* stream);
@@ -132,7 +139,7 @@ int vit_head(vit_handle* h, int microbatch, const void* tokens, float* logits,
  * the normalised class-token features; this variant keeps that scratch in an array that is part
  * of the library itself, so the caller passes only tokens and logits.
  *   - Same arithmetic and same results as vit_head.
- *   - Limit: microbatch * hidden <= VIT_HEAD_STATIC_MAX_FLOATS (2 MiB of floats); anything
+ *   - Limit: microbatch * (1 + extra_tokens) * hidden <= VIT_HEAD_STATIC_MAX_FLOATS (2 MiB of floats); anything
  *     larger returns VIT_ERR_TOO_LARGE and launches nothing.  Every GPU on which the library
  *     is loaded carries the array (2 MiB) until the process exits.
  *   - The first call on each device looks up the array's device address (a runtime query, not

@@ -40,7 +40,7 @@ class VitConfig(Structure):
         ("image_size", c_int32), ("patch_size", c_int32), ("channels", c_int32),
         ("hidden", c_int32), ("layers", c_int32), ("heads", c_int32), ("mlp_dim", c_int32),
         ("num_classes", c_int32), ("ln_eps", c_float), ("dtype", c_int32),
-        ("max_microbatch", c_int32),
+        ("max_microbatch", c_int32), ("extra_tokens", c_int32),
     ]
 
 
@@ -137,7 +137,7 @@ def make_config(shape, dtype=VIT_BF16, max_microbatch=1) -> VitConfig:
     mlp_dim, num_classes, ln_eps attributes."""
     return VitConfig(shape.image_size, shape.patch_size, shape.channels, shape.hidden, shape.layers,
                      shape.heads, shape.mlp_dim, shape.num_classes, float(shape.ln_eps), int(dtype),
-                     int(max_microbatch))
+                     int(max_microbatch), int(getattr(shape, "extra_tokens", 0)))
 
 
 # ---- thin wrappers with the names of the C entry points (raw pointers as ints) ----------------
@@ -311,7 +311,7 @@ class VitModel:
         self.device = torch.device(device)
         self.cfg = make_config(shape, dtype, max_microbatch)
         self.act_dtype = torch.bfloat16 if dtype == VIT_BF16 else torch.float32
-        self.T = (shape.image_size // shape.patch_size) ** 2 + 1
+        self.T = (shape.image_size // shape.patch_size) ** 2 + 1 + int(getattr(shape, "extra_tokens", 0))
         with torch.cuda.device(self.device):
             self.h = vit_create(self.cfg, host_params)
         self._ws = {}

@@ -96,7 +96,7 @@ struct TcParams {
   const float* bias;
   const bf16* residual;   // EPI_BIAS_RESIDUAL
   const float* pos;       // EPI_BIAS_POS
-  int n_patches;
+  int n_patches, first_patch_token;
   bf16* out;
   int ldo;
   int tiles_m, tiles_n;
@@ -245,8 +245,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         const int row = m0 + quarter * 32 + lane;
         const bool row_ok = row < p.M;
         const int img = row / p.n_patches, pt = row - img * p.n_patches;
-        const size_t orow = (size_t)img * (p.n_patches + 1) + 1 + pt;
-        const float* posrow = p.pos + (size_t)(1 + pt) * p.N;
+        const size_t orow = (size_t)img * (p.n_patches + p.first_patch_token) + p.first_patch_token + pt;
+        const float* posrow = p.pos + (size_t)(p.first_patch_token + pt) * p.N;
 #pragma unroll 1
         for (int ch = 0; ch < COLS_PER_WARP / 32; ++ch) {
           const int cl = half * COLS_PER_WARP + ch * 32;
@@ -550,6 +550,7 @@ cudaError_t launch_linear_tc(const LinearArgs& a, int* dev_status, cudaStream_t 
   p.residual = static_cast<const bf16*>(a.residual);
   p.pos = a.pos;
   p.n_patches = a.n_patches > 0 ? a.n_patches : 1;
+  p.first_patch_token = a.first_patch_token > 0 ? a.first_patch_token : 1;
   p.out = static_cast<bf16*>(a.out);
   p.ldo = a.ldo;
   p.tiles_m = tiles_m;

@@ -195,8 +195,9 @@ linear_f32_kernel(LinearArgs p) {
     const float* posrow = nullptr;
     if (p.epilogue == EPI_BIAS_POS) {
       const int img = r / p.n_patches, pt = r % p.n_patches;
-      orow = (size_t)img * (p.n_patches + 1) + 1 + pt;
-      posrow = p.pos + (size_t)(1 + pt) * p.N;
+      const int t0 = p.first_patch_token > 0 ? p.first_patch_token : 1;
+      orow = (size_t)img * (p.n_patches + t0) + t0 + pt;
+      posrow = p.pos + (size_t)(t0 + pt) * p.N;
     }
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
@@ -327,39 +328,45 @@ cudaError_t launch_im2col(const float* pixels, void* cols, int images, int C, in
   return cudaGetLastError();
 }
 
-// Token 0 of every image: cls + pos[0].
+// Special tokens of every image: token 0 = cls + pos[0]; token 1 = dist + pos[1] when the model
+// has a distillation token (n_special = 2).
 template <typename TOut>
-__global__ void cls_rows_kernel(const float* __restrict__ cls, const float* __restrict__ pos,
-                                TOut* __restrict__ tokens, int images, int T, int H) {
+__global__ void cls_rows_kernel(const float* __restrict__ cls, const float* __restrict__ dist,
+                                const float* __restrict__ pos, TOut* __restrict__ tokens, int images,
+                                int T, int H, int n_special) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= images * H) return;
-  const int img = i / H, c = i % H;
-  tokens[(size_t)img * T * H + c] = (TOut)(cls[c] + pos[c]);
+  if (i >= images * n_special * H) return;
+  const int c = i % H, r = (i / H) % n_special, img = i / (H * n_special);
+  const float v = (r == 0 ? cls[c] : dist[c]) + pos[(size_t)r * H + c];
+  tokens[((size_t)img * T + r) * H + c] = (TOut)v;
 }
 
-cudaError_t launch_cls_rows(const float* cls, const float* pos, void* tokens, int images, int T,
-                            int H, bool act_bf16, cudaStream_t s) {
+cudaError_t launch_cls_rows(const float* cls, const float* dist, const float* pos, void* tokens, int images,
+                            int T, int H, bool act_bf16, cudaStream_t s) {
   if (images <= 0) return cudaSuccess;
-  const int threads = 256, blocks = (images * H + threads - 1) / threads;
+  const int n_special = dist ? 2 : 1;
+  const int threads = 256, blocks = (images * n_special * H + threads - 1) / threads;
   if (act_bf16)
-    cls_rows_kernel<bf16><<<blocks, threads, 0, s>>>(cls, pos, (bf16*)tokens, images, T, H);
+    cls_rows_kernel<bf16><<<blocks, threads, 0, s>>>(cls, dist, pos, (bf16*)tokens, images, T, H, n_special);
   else
-    cls_rows_kernel<float><<<blocks, threads, 0, s>>>(cls, pos, (float*)tokens, images, T, H);
+    cls_rows_kernel<float><<<blocks, threads, 0, s>>>(cls, dist, pos, (float*)tokens, images, T, H, n_special);
   return cudaGetLastError();
 }
 
 // ------------------------------------------------------------------------------------------
-// Classification head: (1) LayerNorm of the class token of every image into fp32 features,
-// (2) logits[img, c] = feat[img] . W[c] + bias[c], one warp per class looping over images.
+// Classification head: (1) LayerNorm of the class token (and of the distillation token, if the
+// model has one) of every image into fp32 features, (2) logits[img, c] = feat[img] . W[c] + bias[c],
+// one warp per class looping over images; with two classifiers the mean of the two.
 // ------------------------------------------------------------------------------------------
 template <typename TIn>
 __global__ void head_ln_kernel(const TIn* __restrict__ tokens, const float* __restrict__ g,
                                const float* __restrict__ b, float eps, float* __restrict__ feat,
-                               int images, int T, int H) {
-  const int img = (int)((blockIdx.x * (size_t)blockDim.x + threadIdx.x) >> 5);
+                               int images, int T, int H, int n_special) {
+  const int idx = (int)((blockIdx.x * (size_t)blockDim.x + threadIdx.x) >> 5);   // image * n_special + token
   const int lane = threadIdx.x & 31;
-  if (img >= images) return;
-  const TIn* xr = tokens + (size_t)img * T * H;
+  if (idx >= images * n_special) return;
+  const int img = idx / n_special, r = idx % n_special;
+  const TIn* xr = tokens + ((size_t)img * T + r) * H;
   float sum = 0.f;
   for (int i = lane; i < H; i += 32) sum += (float)xr[i];
   const float mean = warp_sum(sum) / (float)H;
@@ -370,7 +377,7 @@ __global__ void head_ln_kernel(const TIn* __restrict__ tokens, const float* __re
   }
   const float rstd = 1.0f / sqrtf(warp_sum(sq) / (float)H + eps);
   for (int i = lane; i < H; i += 32)
-    feat[(size_t)img * H + i] = ((float)xr[i] - mean) * rstd * g[i] + b[i];
+    feat[(size_t)idx * H + i] = ((float)xr[i] - mean) * rstd * g[i] + b[i];
 }
 
 // One warp per class and group of HEAD_IMGS images: a weight element is loaded once and used
@@ -379,45 +386,51 @@ constexpr int HEAD_IMGS = 8;
 template <typename TW>
 __global__ void __launch_bounds__(256)
 head_logits_kernel(const float* __restrict__ feat, const TW* __restrict__ W,
-                   const float* __restrict__ bias, float* __restrict__ logits, int images, int H,
+                   const float* __restrict__ bias, const TW* __restrict__ W2,
+                   const float* __restrict__ bias2, float* __restrict__ logits, int images, int H,
                    int classes) {
   const int c = blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   const int img0 = blockIdx.y * HEAD_IMGS;
   if (c >= classes) return;
-  const TW* wr = W + (size_t)c * H;
+  const int n_special = W2 ? 2 : 1;
   float acc[HEAD_IMGS];
 #pragma unroll
   for (int j = 0; j < HEAD_IMGS; ++j) acc[j] = 0.f;
-  for (int i = lane; i < H; i += 32) {
-    const float w = (float)wr[i];
+  for (int r = 0; r < n_special; ++r) {
+    const TW* wr = (r == 0 ? W : W2) + (size_t)c * H;
+    for (int i = lane; i < H; i += 32) {
+      const float w = (float)wr[i];
 #pragma unroll
-    for (int j = 0; j < HEAD_IMGS; ++j) {
-      const int img = img0 + j < images ? img0 + j : images - 1;
-      acc[j] = fmaf(feat[(size_t)img * H + i], w, acc[j]);
+      for (int j = 0; j < HEAD_IMGS; ++j) {
+        const int img = img0 + j < images ? img0 + j : images - 1;
+        acc[j] = fmaf(feat[((size_t)img * n_special + r) * H + i], w, acc[j]);
+      }
     }
   }
-  const float bc = bias[c];
+  const float bc = W2 ? bias[c] + bias2[c] : bias[c];
+  const float scale = W2 ? 0.5f : 1.0f;
 #pragma unroll
   for (int j = 0; j < HEAD_IMGS; ++j) {
     const float s = warp_sum(acc[j]);
-    if (lane == 0 && img0 + j < images) logits[(size_t)(img0 + j) * classes + c] = s + bc;
+    if (lane == 0 && img0 + j < images) logits[(size_t)(img0 + j) * classes + c] = (s + bc) * scale;
   }
 }
 
 cudaError_t launch_head(const void* tokens, const float* g, const float* b, float eps,
-                        const void* W, const float* bias, float* feat, float* logits, int images,
-                        int T, int H, int classes, bool act_bf16, cudaStream_t s) {
+                        const void* W, const float* bias, const void* W2, const float* bias2, float* feat,
+                        float* logits, int images, int T, int H, int classes, bool act_bf16, cudaStream_t s) {
   if (images <= 0) return cudaSuccess;
+  const int n_special = W2 ? 2 : 1;
   const int threads = 256;
-  const unsigned b1 = (unsigned)(((size_t)images * 32 + threads - 1) / threads);
+  const unsigned b1 = (unsigned)(((size_t)images * n_special * 32 + threads - 1) / threads);
   const dim3 b2((unsigned)((classes + 7) / 8), (unsigned)((images + HEAD_IMGS - 1) / HEAD_IMGS));
   if (act_bf16) {
-    head_ln_kernel<bf16><<<b1, threads, 0, s>>>((const bf16*)tokens, g, b, eps, feat, images, T, H);
-    head_logits_kernel<bf16><<<b2, threads, 0, s>>>(feat, (const bf16*)W, bias, logits, images, H, classes);
+    head_ln_kernel<bf16><<<b1, threads, 0, s>>>((const bf16*)tokens, g, b, eps, feat, images, T, H, n_special);
+    head_logits_kernel<bf16><<<b2, threads, 0, s>>>(feat, (const bf16*)W, bias, (const bf16*)W2, bias2, logits, images, H, classes);
   } else {
-    head_ln_kernel<float><<<b1, threads, 0, s>>>((const float*)tokens, g, b, eps, feat, images, T, H);
-    head_logits_kernel<float><<<b2, threads, 0, s>>>(feat, (const float*)W, bias, logits, images, H, classes);
+    head_ln_kernel<float><<<b1, threads, 0, s>>>((const float*)tokens, g, b, eps, feat, images, T, H, n_special);
+    head_logits_kernel<float><<<b2, threads, 0, s>>>(feat, (const float*)W, bias, (const float*)W2, bias2, logits, images, H, classes);
   }
   return cudaGetLastError();
 }
@@ -437,7 +450,8 @@ float* g_static_ptr[kMaxDevices] = {};
 }  // namespace
 
 cudaError_t launch_head_static(const void* tokens, const float* g, const float* b, float eps,
-                               const void* W, const float* bias, float* logits, int images, int T,
+                               const void* W, const float* bias, const void* W2, const float* bias2,
+                               float* logits, int images, int T,
                                int H, int classes, bool act_bf16, cudaStream_t s) {
   int dev = -1;
   cudaError_t e = cudaGetDevice(&dev);
@@ -457,7 +471,7 @@ cudaError_t launch_head_static(const void* tokens, const float* g, const float* 
   }
   // Every feature the logits kernel reads is written by the LayerNorm kernel of the same call
   // first, so nothing in the array has to start at zero.
-  return launch_head(tokens, g, b, eps, W, bias, scratch, logits, images, T, H, classes, act_bf16, s);
+  return launch_head(tokens, g, b, eps, W, bias, W2, bias2, scratch, logits, images, T, H, classes, act_bf16, s);
 }
 
 }  // namespace vit

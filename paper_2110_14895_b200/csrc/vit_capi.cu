@@ -31,18 +31,20 @@ bool config_ok(const vit_config* c) {
   if (c->layers <= 0 || c->num_classes <= 0 || c->max_microbatch <= 0) return false;
   if (c->dtype != VIT_BF16 && c->dtype != VIT_FP32) return false;
   if (!(c->ln_eps >= 0.f)) return false;
+  if (c->extra_tokens != 0 && c->extra_tokens != 1) return false;
   const int g = c->image_size / c->patch_size;
-  if (g * g + 1 > 512) return false;
+  if (g * g + 1 + c->extra_tokens > 512) return false;
   return true;
 }
 
 struct Shape {
-  int T, Np, d, Kpe, Kpad;
+  int T, Np, d, Kpe, Kpad, X;      // X: special tokens besides the class token
   size_t H, F, C;
   explicit Shape(const vit_config& c) {
     const int g = c.image_size / c.patch_size;
     Np = g * g;
-    T = Np + 1;
+    X = c.extra_tokens;
+    T = Np + 1 + X;
     d = c.hidden / c.heads;
     Kpe = c.channels * c.patch_size * c.patch_size;
     Kpad = (Kpe + 63) / 64 * 64;
@@ -52,11 +54,11 @@ struct Shape {
 
 size_t param_count(const vit_config& c) {
   const Shape s(c);
-  size_t n = s.H * s.Kpe + s.H + s.H + (size_t)s.T * s.H;
+  size_t n = s.H * s.Kpe + s.H + s.H + (size_t)s.X * s.H + (size_t)s.T * s.H;
   const size_t per_layer = 2 * s.H + 3 * s.H * s.H + 3 * s.H + s.H * s.H + s.H + 2 * s.H +
                            s.F * s.H + s.F + s.H * s.F + s.H;
   n += per_layer * c.layers;
-  n += 2 * s.H + s.C * s.H + s.C;
+  n += 2 * s.H + (1 + (size_t)s.X) * (s.C * s.H + s.C);
   return n;
 }
 
@@ -74,7 +76,7 @@ size_t embed_ws_bytes(const vit_config& c, int mb) {
 }
 size_t head_ws_bytes(const vit_config& c, int mb) {
   const Shape s(c);
-  return align_up((size_t)mb * s.H * sizeof(float), 256);
+  return align_up((size_t)mb * (1 + s.X) * s.H * sizeof(float), 256);
 }
 size_t call_ws_bytes(const vit_config& c, int mb) {
   size_t w = stage_ws_bytes(c, mb);
@@ -265,6 +267,7 @@ int vit_create(const vit_config* cfg, const float* host_params, size_t n_params,
   const size_t i_pw = add(s.H, s.Kpe, s.Kpad, true);
   const size_t i_pb = add(1, s.H, s.H, false);
   const size_t i_cls = add(1, s.H, s.H, false);
+  const size_t i_dist = s.X ? add(1, s.H, s.H, false) : 0;
   const size_t i_pos = add(s.T, s.H, s.H, false);
   std::vector<size_t> li(L);
   for (int l = 0; l < L; ++l) {
@@ -285,6 +288,8 @@ int vit_create(const vit_config* cfg, const float* host_params, size_t n_params,
   const size_t i_lnfb = add(1, s.H, s.H, false);
   const size_t i_hw = add(s.C, s.H, s.H, true);
   const size_t i_hb = add(1, s.C, s.C, false);
+  const size_t i_hdw = s.X ? add(s.C, s.H, s.H, true) : 0;
+  const size_t i_hdb = s.X ? add(1, s.C, s.C, false) : 0;
   if (src != n_params) return VIT_ERR_INVALID_ARG;
   const size_t blob_bytes = dst;
 
@@ -330,7 +335,7 @@ int vit_create(const vit_config* cfg, const float* host_params, size_t n_params,
   const uint8_t* B = static_cast<const uint8_t*>(dev_blob);
   auto fp = [&](size_t i) { return reinterpret_cast<const float*>(B + items[i].dst); };
   auto vp = [&](size_t i) { return static_cast<const void*>(B + items[i].dst); };
-  h->patch_W = vp(i_pw); h->patch_b = fp(i_pb); h->cls = fp(i_cls); h->pos = fp(i_pos);
+  h->patch_W = vp(i_pw); h->patch_b = fp(i_pb); h->cls = fp(i_cls); h->dist = s.X ? fp(i_dist) : nullptr; h->pos = fp(i_pos);
   h->layers = new LayerWeights[L];
   for (int l = 0; l < L; ++l) {
     const size_t b = li[l];
@@ -340,6 +345,7 @@ int vit_create(const vit_config* cfg, const float* host_params, size_t n_params,
     w.W1 = vp(b + 8); w.b1 = fp(b + 9); w.W2 = vp(b + 10); w.b2 = fp(b + 11);
   }
   h->lnf_g = fp(i_lnfg); h->lnf_b = fp(i_lnfb); h->head_W = vp(i_hw); h->head_b = fp(i_hb);
+  h->head_dist_W = s.X ? vp(i_hdw) : nullptr; h->head_dist_b = s.X ? fp(i_hdb) : nullptr;
   *out = h;
   return VIT_OK;
 }
@@ -370,11 +376,11 @@ int vit_patch_embed(vit_handle* h, int mb, const float* pixels, void* tokens_out
   a.w = h->patch_W; a.ldw = h->patch_k_pad;
   a.bias = h->patch_b;
   a.epilogue = EPI_BIAS_POS;
-  a.pos = h->pos; a.n_patches = h->n_patches;
+  a.pos = h->pos; a.n_patches = h->n_patches; a.first_patch_token = 1 + c.extra_tokens;
   a.out = tokens_out; a.ldo = c.hidden;
   st = linear(h, VIT_PROF_EMBED, a, s);
   if (st != VIT_OK) return st;
-  VIT_LAUNCH(h, VIT_PROF_EMBED, launch_cls_rows(h->cls, h->pos, tokens_out, mb, h->T, c.hidden, b16, s));
+  VIT_LAUNCH(h, VIT_PROF_EMBED, launch_cls_rows(h->cls, h->dist, h->pos, tokens_out, mb, h->T, c.hidden, b16, s));
   return VIT_OK;
 }
 
@@ -446,7 +452,7 @@ int vit_head(vit_handle* h, int mb, const void* tokens, float* logits, void* ws,
   const vit_config& c = h->cfg;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   VIT_LAUNCH(h, VIT_PROF_HEAD, launch_head(tokens, h->lnf_g, h->lnf_b, c.ln_eps, h->head_W, h->head_b,
-                                           static_cast<float*>(ws), logits, mb, h->T, c.hidden,
+                                           h->head_dist_W, h->head_dist_b, static_cast<float*>(ws), logits, mb, h->T, c.hidden,
                                            c.num_classes, c.dtype == VIT_BF16, s));
   h->launches.fetch_add(1, std::memory_order_relaxed);   // the head is two kernels
   return VIT_OK;
@@ -456,10 +462,10 @@ int vit_head_static(vit_handle* h, int mb, const void* tokens, float* logits, vo
   if (!h || mb < 1 || mb > h->cfg.max_microbatch || !on_own_device(h)) return VIT_ERR_INVALID_ARG;
   if (!tokens || !logits || misaligned(tokens) || misaligned(logits)) return VIT_ERR_INVALID_ARG;
   const vit_config& c = h->cfg;
-  if ((size_t)mb * (size_t)c.hidden > (size_t)VIT_HEAD_STATIC_MAX_FLOATS) return VIT_ERR_TOO_LARGE;
+  if ((size_t)mb * (size_t)(1 + c.extra_tokens) * (size_t)c.hidden > (size_t)VIT_HEAD_STATIC_MAX_FLOATS) return VIT_ERR_TOO_LARGE;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   VIT_LAUNCH(h, VIT_PROF_HEAD, launch_head_static(tokens, h->lnf_g, h->lnf_b, c.ln_eps, h->head_W,
-                                                  h->head_b, logits, mb, h->T, c.hidden,
+                                                  h->head_b, h->head_dist_W, h->head_dist_b, logits, mb, h->T, c.hidden,
                                                   c.num_classes, c.dtype == VIT_BF16, s));
   h->launches.fetch_add(1, std::memory_order_relaxed);   // the head is two kernels
   return VIT_OK;

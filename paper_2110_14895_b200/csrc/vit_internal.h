@@ -20,7 +20,7 @@ enum Epilogue : int {
   EPI_BIAS_GELU = 1,     // out = gelu(acc + bias), erf form
   EPI_BIAS_RESIDUAL = 2, // out = acc + bias + residual[row, col]
   EPI_BIAS_POS = 3       // patch embed: row r of the GEMM is patch r % n_patches of image r / n_patches;
-                         // out[image*T + 1 + patch, col] = acc + bias + pos[1 + patch, col]
+                         // out[image*T + t0 + patch, col] = acc + bias + pos[t0 + patch, col], T = t0 + n_patches
 };
 
 struct LinearArgs {
@@ -34,6 +34,7 @@ struct LinearArgs {
   const void* residual;   // EPI_BIAS_RESIDUAL: [M, N] stride ldo; may alias out
   const float* pos;       // EPI_BIAS_POS: [T, N] fp32
   int n_patches;          // EPI_BIAS_POS
+  int first_patch_token;  // EPI_BIAS_POS: t0, the number of special tokens before the patches
   void* out;              // activation type, row stride ldo
   int ldo;
   int tiling;             // bf16 tensor-core kernel: TILING_AUTO (shape-only cost model) or a forced tiling
@@ -57,10 +58,10 @@ struct Handle {
   void* dev_blob;                    // every parameter, one allocation
   size_t dev_blob_bytes;
   const void* patch_W;               // [H, patch_k_pad]
-  const float *patch_b, *cls, *pos;
+  const float *patch_b, *cls, *dist, *pos;          // dist: distillation token (nullptr without one)
   LayerWeights* layers;              // host array [L]
-  const float *lnf_g, *lnf_b, *head_b;
-  const void* head_W;                // [classes, H]
+  const float *lnf_g, *lnf_b, *head_b, *head_dist_b;
+  const void *head_W, *head_dist_W;  // [classes, H]; head_dist_*: second classifier (nullptr without a distillation token)
   int* dev_status;                   // device: [0] status word (0 = ok), [1] snapshot slot of vit_check_status
   std::mutex status_mutex;
   std::atomic<uint64_t> launches;
@@ -88,15 +89,20 @@ cudaError_t launch_attention_f32(const float* qkv, float* out, int images, int T
 // book-ends, both families (act_bf16 selects the element type)
 cudaError_t launch_im2col(const float* pixels, void* cols, int images, int C, int S, int P,
                           int k_pad, bool act_bf16, cudaStream_t s);
-cudaError_t launch_cls_rows(const float* cls, const float* pos, void* tokens, int images, int T,
-                            int H, bool act_bf16, cudaStream_t s);
+// special tokens: token 0 = cls + pos[0]; token 1 = dist + pos[1] when dist != nullptr
+cudaError_t launch_cls_rows(const float* cls, const float* dist, const float* pos, void* tokens, int images,
+                            int T, int H, bool act_bf16, cudaStream_t s);
+// W2 / bias2 != nullptr: second classifier on token 1, logits = mean of the two (feat_scratch then
+// holds two feature rows per image)
 cudaError_t launch_head(const void* tokens, const float* g, const float* b, float eps,
-                        const void* W, const float* bias, float* feat_scratch, float* logits,
+                        const void* W, const float* bias, const void* W2, const float* bias2,
+                        float* feat_scratch, float* logits,
                         int images, int T, int H, int classes, bool act_bf16, cudaStream_t s);
 
 // head with the feature scratch in a fixed device array of VIT_HEAD_STATIC_MAX_FLOATS floats
 cudaError_t launch_head_static(const void* tokens, const float* g, const float* b, float eps,
-                               const void* W, const float* bias, float* logits, int images, int T,
+                               const void* W, const float* bias, const void* W2, const float* bias2,
+                               float* logits, int images, int T,
                                int H, int classes, bool act_bf16, cudaStream_t s);
 
 cudaError_t launch_wait_probe(long long limit_cycles, int* dev_status, cudaStream_t s);

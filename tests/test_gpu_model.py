@@ -156,6 +156,49 @@ def test_small16_batch32_two_microbatches_three_stages():
     m.close()
 
 
+# ---------------------------------------------------------------------------------------------
+# The compressed (distilled) family: a distillation token after the class token (198 tokens) and a
+# second classifier; tiny / small / base dimensions.
+@pytest.mark.parametrize("dtype_name", ["bf16", "fp32"])
+def test_distilled_tiny_intermediate_tensors_and_logits_match_oracle(dtype_name):
+    vit = _vit()
+    dtype = vit.VIT_BF16 if dtype_name == "bf16" else vit.VIT_FP32
+    shape = vitgen.preset("deit_tiny16").with_(layers=2)
+    vit, m, params = _model(shape, dtype, 3, seed=7, ln_affine=True, bf16_weights=dtype_name == "bf16")
+    assert m.T == 198
+    pix = vitgen.make_pixels(shape, 3, seed=7)
+    x = m.patch_embed(torch.from_numpy(pix).cuda())
+    m.check()
+    want = O.patch_embed(params, shape, pix)
+    got = x.float().cpu().numpy()
+    tol = 1e-5 if dtype_name == "fp32" else 2.0 ** -8
+    assert np.abs(got - want).max() <= tol * np.abs(want).max() + (3e-3 if dtype_name == "bf16" else 0)
+    # the two special rows exactly as defined
+    assert np.abs(got[:, :2] - want[:, :2]).max() <= tol * np.abs(want[:, :2]).max()
+    y = m.run_stage(0, 2, x)
+    logits = m.head(y)
+    m.check()
+    want_y = O.run_stage(params, shape, 0, 2, want)
+    want_l = O.head(params, shape, want_y)
+    ok, msg = logits_within_tolerance(logits.cpu().numpy(), want_l, 1e-3 if dtype_name == "fp32" else 2e-2)
+    assert ok, msg
+    # the head on the oracle's own tokens isolates the two-classifier mean from upstream error
+    yt = torch.from_numpy(want_y.astype(np.float32)).cuda().to(m.act_dtype)
+    l2 = m.head(yt).cpu().numpy()
+    want_l2 = O.head(params, shape, yt.float().cpu().numpy().astype(np.float64))
+    assert np.abs(l2 - want_l2).max() <= 1e-4 * max(1.0, np.abs(want_l2).max())
+    m.close()
+
+
+@pytest.mark.parametrize("name,batch,mb", [("deit_tiny16", 8, 4), ("deit_small16", 32, 16), ("deit_base16", 32, 16)])
+def test_distilled_models_pipeline_matches_oracle(name, batch, mb):
+    sample = [0, mb - 1, mb, batch - 1]
+    _, m, pix, got = _pipeline_vs_oracle(name, batch, mb, vitgen.equal_partition(4, 12), 2, sample)
+    one = m.forward(torch.from_numpy(pix[mb:2 * mb]).cuda())
+    assert np.array_equal(one.cpu().numpy(), got[mb:2 * mb])       # staged == single call, bit for bit
+    m.close()
+
+
 def test_base16_host_buffers_pipeline():
     _, m, _, _ = _pipeline_vs_oracle("base16", 8, 4, vitgen.equal_partition(4, 12), 2, [0, 3, 4, 7], host=True)
     m.close()

@@ -40,6 +40,20 @@ def test_head_static_matches_head_on_two_calls_in_a_row():
     m.close()
 
 
+def test_head_static_with_distillation_token_matches_head():
+    """Two feature rows per image (class and distillation token) go through the fixed array."""
+    shape = vitgen.preset("deit_tiny16").with_(layers=1)
+    vit, m = _model(shape, 6)
+    tokens = torch.randn((6, m.T, shape.hidden), device="cuda").to(torch.bfloat16)
+    want = m.head(tokens)
+    for _ in range(2):
+        got = torch.full_like(want, float("nan"))
+        vit.vit_head_static(m.h, 6, tokens.data_ptr(), got.data_ptr())
+        m.check()
+        assert torch.equal(got, want)
+    m.close()
+
+
 def test_head_static_fp32_mode_matches_head():
     shape = vitgen.preset("tiny16").with_(layers=1)
     vit, m = _model(shape, 3, dtype=1)

@@ -288,6 +288,54 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+def run_stage_per_gpu(args, vit, torch, dist, dev, rank, world):
+    """One pipeline stage per GPU (strong scaling: the batch is fixed, the layers are spread).
+    Every rank holds the whole parameter set and runs its own layer range; activations travel
+    rank to rank by NCCL send/receive into the receiver's own buffers."""
+    from paper_2110_14895_b200 import pipeline as PL
+    preset, batch, mb, _ = WORKLOADS[args.workload]
+    mb = min(mb, 32)
+    shape = vitgen.preset(preset)
+    if world > shape.layers:
+        raise SystemExit("more GPUs than layers")
+    _, layers = PL.plan_stages([1.0] * shape.layers, world, act_bytes=1.0, link_bytes_per_s=1e30)
+    if len(layers) != world:
+        raise SystemExit("the partitioner used fewer stages than GPUs")
+    lb, le = PL.stage_ranges(layers)[rank]
+    _, blob = vitgen.make_params(shape, seed=0)
+    model = vit.VitModel(shape, blob, vit.VIT_BF16, mb, device=dev)
+    del blob
+    pipe = PL.StagePipeline(PL.VitStageExecutor(model, lb, le, rank == 0, rank == world - 1), dist, mb)
+    pix = torch.from_numpy(vitgen.make_pixels(shape, batch, seed=0)).to(dev) if rank == 0 else None
+    logits = torch.empty((batch, shape.num_classes), dtype=torch.float32, device=dev) if rank == world - 1 else None
+    for _ in range(args.warmup):
+        pipe.run(batch, mb, pixels=pix, logits=logits)
+    torch.cuda.synchronize(dev)
+    dist.barrier()
+    torch.cuda.synchronize(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        pipe.run(batch, mb, pixels=pix, logits=logits)
+    e1.record()
+    torch.cuda.synchronize(dev)
+    dist.barrier()
+    ms = max_over_ranks(e0.elapsed_time(e1), dist, dev) / args.steps
+    model.check()
+    if rank == 0:
+        total_flops = flops_per_image(shape)[0]
+        value = batch / (ms / 1e3)
+        print(json.dumps({
+            "metric": "images/sec", "value": value, "unit": "images/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "strong",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"ViT-{preset} forward, batch {batch}, microbatch {mb}, one stage per GPU, "
+                                   f"layers per stage {layers}", "global_batch": batch,
+                       "parallelism": f"pipeline pp{world}", "l2": "activations and weights per layer exceed L2"},
+            "tflops": value * total_flops / 1e12}), flush=True)
+    model.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -299,6 +347,9 @@ def main():
     ap.add_argument("--no-extra-workloads", action="store_true",
                     help="skip the brief ViT-L/16 and ViT-B/16 measurements reported under 'workloads'")
     ap.add_argument("--streams", type=int, default=0, help="streams for the stage runner (0 = min(4, microbatches))")
+    ap.add_argument("--mode", default="replicas", choices=["replicas", "pipeline"],
+                    help="N > 1 only: independent replicas (default), or one pipeline stage per GPU with "
+                         "point-to-point hand-off of the activations (the paper's runtime)")
     ap.add_argument("--sweep", action="store_true",
                     help="also run the microbatch sweep (sizes 1..256, 4 stages, streams) and add it as 'sweep'")
     args = ap.parse_args()
@@ -319,6 +370,11 @@ def main():
     dev = torch.device("cuda", local)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+
+    if args.mode == "pipeline" and world > 1:
+        run_stage_per_gpu(args, vit, torch, dist, dev, rank, world)
+        dist.destroy_process_group()
+        return
 
     preset, batch, mb, n_stages = WORKLOADS[args.workload]
     shape = vitgen.preset(preset)

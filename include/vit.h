@@ -114,7 +114,9 @@ int vit_patch_embed(vit_handle* h, int microbatch, const float* pixels, void* to
  * consecutive layers, the output of stage i is the input of stage i+1, and
  * Y = T_k(...T_1(X))).  Applies layers [layer_begin, layer_end) to `in`, writes `out`.
  * Each layer is x += Wo.attention(LN1(x).Wqkv^T + bqkv) + bo;  x += W2.gelu(W1.LN2(x) + b1) + b2
- * (Section 2.1: self-attention, MLP, two layer normalisations, residual connections).
+ * (Section 2.1: self-attention, MLP, two layer normalisations, residual connections).  In bf16
+ * mode the two layer normalisations are applied inside the QKV and fc1 products (row statistics
+ * from a small kernel, gain and shift folded into the weights at vit_create).
  *   in, out: dev, activations [microbatch, T, H]; in == out is allowed (in place), any other
  *     overlap is INVALID_ARG.
  * Running [a,b) then [b,c) gives bit-identical results to one call on [a,c). */
@@ -275,6 +277,18 @@ enum { VIT_TILING_AUTO = 0, VIT_TILING_128x128 = 1, VIT_TILING_128x256 = 2, VIT_
 int vit_op_linear_tiled(vit_handle* h, int dtype, int M, int N, int K, const void* a, const void* w,
                         const float* bias, int epilogue, const void* residual, void* out, int tiling,
                         void* stream);
+
+/* The two halves of the LayerNorm that vit_run_stage folds into its QKV and fc1 products in bf16
+ * mode (the normalised activations are never written to memory):
+ *   vit_op_rowstats: stats[2 r] = mean of row r of x (bf16 [rows, cols]), stats[2 r + 1] =
+ *     1 / sqrt(biased variance + eps); stats is fp32 [rows, 2].
+ *   vit_op_linear_ln: out[m,n] = f(stats[m].rstd * (a[m,:] . wg[n,:] - stats[m].mean * c1[n]) + c0[n]),
+ *     f = identity or erf-GELU.  With wg[n,k] = gain[k] w[n,k], c1[n] = sum_k wg[n,k] and
+ *     c0[n] = bias[n] + sum_k shift[k] w[n,k] this equals f(LayerNorm(a)[m,:] . w[n,:] + bias[n]).
+ *     a, wg, out bf16; c1, c0 fp32 [N]; `tiling` as in vit_op_linear_tiled. */
+int vit_op_rowstats(vit_handle* h, int rows, int cols, const void* x, float eps, float* stats, void* stream);
+int vit_op_linear_ln(vit_handle* h, int M, int N, int K, const void* a, const float* stats, const void* wg,
+                     const float* c1, const float* c0, int gelu, void* out, int tiling, void* stream);
 
 /* Multi-head self-attention for `images` sequences of T tokens: qkv [images*T, 3*heads*d]
  * (column blocks Q, K, V; head-major inside each), out [images*T, heads*d];

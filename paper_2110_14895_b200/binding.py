@@ -28,7 +28,7 @@ EXPORTS = [
     "vit_param_count", "vit_workspace_bytes", "vit_pipeline_workspace_bytes", "vit_create",
     "vit_destroy", "vit_patch_embed", "vit_run_stage", "vit_head", "vit_run_pipeline",
     "vit_run_pipeline_host", "vit_run_pipeline_grouped", "vit_check_status", "vit_launch_count", "vit_status_string",
-    "vit_op_layernorm", "vit_op_linear", "vit_op_linear_tiled", "vit_op_attention", "vit_profile_enable",
+    "vit_op_layernorm", "vit_op_linear", "vit_op_linear_tiled", "vit_op_attention", "vit_op_rowstats", "vit_op_linear_ln", "vit_profile_enable",
     "vit_profile_collect", "vit_head_static", "vit_partition", "vit_partition_categories",
     "vit_debug_wait_probe",
 ]
@@ -104,6 +104,11 @@ def lib():
     L.vit_op_linear.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p]
     L.vit_op_linear_tiled.restype = c_int
     L.vit_op_linear_tiled.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_int, c_void_p]
+    L.vit_op_rowstats.restype = c_int
+    L.vit_op_rowstats.argtypes = [c_void_p, c_int, c_int, c_void_p, c_float, c_void_p, c_void_p]
+    L.vit_op_linear_ln.restype = c_int
+    L.vit_op_linear_ln.argtypes = [c_void_p, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p,
+                                   c_int, c_void_p, c_int, c_void_p]
     L.vit_op_attention.restype = c_int
     L.vit_op_attention.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_void_p, c_void_p, c_void_p]
     L.vit_head_static.restype = c_int
@@ -294,6 +299,15 @@ def vit_op_linear(h, dtype, M, N, K, a, w, bias, epilogue, residual, out, stream
 def vit_op_linear_tiled(h, dtype, M, N, K, a, w, bias, epilogue, residual, out, tiling, stream=0):
     _check(lib().vit_op_linear_tiled(h, dtype, M, N, K, a, w, bias, epilogue, residual, out, tiling, stream),
            "vit_op_linear_tiled")
+
+
+def vit_op_rowstats(h, rows, cols, x, eps, stats, stream=0):
+    _check(lib().vit_op_rowstats(h, rows, cols, x, eps, stats, stream), "vit_op_rowstats")
+
+
+def vit_op_linear_ln(h, M, N, K, a, stats, wg, c1, c0, gelu, out, tiling=0, stream=0):
+    _check(lib().vit_op_linear_ln(h, M, N, K, a, stats, wg, c1, c0, 1 if gelu else 0, out, tiling, stream),
+           "vit_op_linear_ln")
 
 
 def vit_op_attention(h, dtype, images, T, heads, d, qkv, out, stream=0):

@@ -96,6 +96,8 @@ struct TcParams {
   const float* bias;
   const bf16* residual;   // EPI_BIAS_RESIDUAL
   const float* pos;       // EPI_BIAS_POS
+  const float2* ln_stats; // EPI_LN_*
+  const float* ln_c1;     // EPI_LN_*
   int n_patches, first_patch_token;
   bf16* out;
   int ldo;
@@ -314,18 +316,33 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
           tmem_ld32(taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
           tmem_ld_wait();
           float v[64];
+          constexpr bool LN = EPI == EPI_LN_BIAS || EPI == EPI_LN_BIAS_GELU;
+          float2 nmean = make_float2(0.f, 0.f), rstd = make_float2(1.f, 1.f);
+          if (LN) {                                  // this thread's row: lane = row of the accumulator
+            const float2 st = (row0 + lane < p.M) ? __ldg(p.ln_stats + row0 + lane) : make_float2(0.f, 1.f);
+            nmean = make_float2(-st.x, -st.x);
+            rstd = make_float2(st.y, st.y);
+          }
 #pragma unroll
           for (int g = 0; g < 16; ++g) {
-            const float4 b = (c0 + 4 * g < p.N) ? __ldg(reinterpret_cast<const float4*>(p.bias + c0) + g)
-                                                : make_float4(0.f, 0.f, 0.f, 0.f);
-            const float2 lo = __fadd2_rn(make_float2(__uint_as_float(r[4 * g + 0]), __uint_as_float(r[4 * g + 1])), make_float2(b.x, b.y));
-            const float2 hi = __fadd2_rn(make_float2(__uint_as_float(r[4 * g + 2]), __uint_as_float(r[4 * g + 3])), make_float2(b.z, b.w));
+            const bool in = c0 + 4 * g < p.N;
+            const float4 b = in ? __ldg(reinterpret_cast<const float4*>(p.bias + c0) + g) : make_float4(0.f, 0.f, 0.f, 0.f);
+            float2 lo = make_float2(__uint_as_float(r[4 * g + 0]), __uint_as_float(r[4 * g + 1]));
+            float2 hi = make_float2(__uint_as_float(r[4 * g + 2]), __uint_as_float(r[4 * g + 3]));
+            if (LN) {
+              const float4 c1 = in ? __ldg(reinterpret_cast<const float4*>(p.ln_c1 + c0) + g) : make_float4(0.f, 0.f, 0.f, 0.f);
+              lo = __ffma2_rn(rstd, __ffma2_rn(nmean, make_float2(c1.x, c1.y), lo), make_float2(b.x, b.y));
+              hi = __ffma2_rn(rstd, __ffma2_rn(nmean, make_float2(c1.z, c1.w), hi), make_float2(b.z, b.w));
+            } else {
+              lo = __fadd2_rn(lo, make_float2(b.x, b.y));
+              hi = __fadd2_rn(hi, make_float2(b.z, b.w));
+            }
             v[4 * g + 0] = lo.x;
             v[4 * g + 1] = lo.y;
             v[4 * g + 2] = hi.x;
             v[4 * g + 3] = hi.y;
           }
-          if (EPI == EPI_BIAS_GELU) {
+          if (EPI == EPI_BIAS_GELU || EPI == EPI_LN_BIAS_GELU) {
 #pragma unroll
             for (int e = 0; e < 64; e += 2) {
               const float2 y = gelu_erf2(make_float2(v[e], v[e + 1]));
@@ -452,6 +469,8 @@ cudaError_t launch_bn(int epi, const Maps& m, const TcParams& p, cudaStream_t s)
     case EPI_BIAS_GELU: return launch_variant<BN, EPI_BIAS_GELU, CTAS>(m, p, s);
     case EPI_BIAS_RESIDUAL: return launch_variant<BN, EPI_BIAS_RESIDUAL, CTAS>(m, p, s);
     case EPI_BIAS_POS: return launch_variant<BN, EPI_BIAS_POS, CTAS>(m, p, s);
+    case EPI_LN_BIAS: return launch_variant<BN, EPI_LN_BIAS, CTAS>(m, p, s);
+    case EPI_LN_BIAS_GELU: return launch_variant<BN, EPI_LN_BIAS_GELU, CTAS>(m, p, s);
   }
   return cudaErrorInvalidValue;
 }
@@ -549,6 +568,9 @@ cudaError_t launch_linear_tc(const LinearArgs& a, int* dev_status, cudaStream_t 
   p.bias = a.bias;
   p.residual = static_cast<const bf16*>(a.residual);
   p.pos = a.pos;
+  p.ln_stats = a.ln_stats;
+  p.ln_c1 = a.ln_c1;
+  if ((a.epilogue == EPI_LN_BIAS || a.epilogue == EPI_LN_BIAS_GELU) && (!a.ln_stats || !a.ln_c1)) return cudaErrorInvalidValue;
   p.n_patches = a.n_patches > 0 ? a.n_patches : 1;
   p.first_patch_token = a.first_patch_token > 0 ? a.first_patch_token : 1;
   p.out = static_cast<bf16*>(a.out);

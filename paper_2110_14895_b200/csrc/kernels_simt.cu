@@ -119,6 +119,82 @@ cudaError_t launch_layernorm_bf16(const bf16* x, const float* g, const float* b,
   return err;
 }
 
+// ------------------------------------------------------------------------------------------
+// LayerNorm statistics only: stats[row] = (mean, 1 / sqrt(biased variance + eps)).  Same warp-
+// per-row scheme as the kernel above (128-bit loads, the row in registers, two-pass variance,
+// shuffle reductions); the normalisation itself is applied by the consumer (the QKV and fc1
+// GEMMs fold it into their epilogue), so nothing but 8 bytes per row is written.
+// ------------------------------------------------------------------------------------------
+template <int NCH>
+__global__ void __launch_bounds__(256)
+rowstats_bf16_kernel(const bf16* __restrict__ x, float eps, float2* __restrict__ stats, int rows, int cols) {
+  const int row = (int)((blockIdx.x * (size_t)blockDim.x + threadIdx.x) >> 5);
+  const int lane = threadIdx.x & 31;
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (row >= rows) return;
+  const int nvec = cols >> 3;
+  const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)row * cols);
+  uint4 u[NCH];
+#pragma unroll
+  for (int i = 0; i < NCH; ++i) {
+    const int idx = lane + 32 * i;
+    u[i] = idx < nvec ? __ldg(xr + idx) : make_uint4(0, 0, 0, 0);
+  }
+  float v[NCH][8];
+  float sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < NCH; ++i) {
+    const uint32_t w[4] = {u[i].x, u[i].y, u[i].z, u[i].w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      v[i][2 * e] = __uint_as_float(w[e] << 16);
+      v[i][2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+      sum += v[i][2 * e] + v[i][2 * e + 1];
+    }
+  }
+  const float mean = warp_sum(sum) / (float)cols;
+  float sq = 0.f;
+#pragma unroll
+  for (int i = 0; i < NCH; ++i) {
+    if (lane + 32 * i < nvec) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const float c = v[i][e] - mean;
+        sq = fmaf(c, c, sq);
+      }
+    }
+  }
+  const float rstd = 1.0f / sqrtf(warp_sum(sq) / (float)cols + eps);
+  if (lane == 0) stats[row] = make_float2(mean, rstd);
+}
+
+cudaError_t launch_rowstats_bf16(const bf16* x, float eps, float2* stats, int rows, int cols, cudaStream_t s) {
+  if (rows <= 0) return cudaSuccess;
+  if (cols % 8 != 0 || cols > 8 * 256) return cudaErrorInvalidValue;
+  const int nch = (cols / 8 + 31) / 32;
+  const int threads = 256;
+  const unsigned blocks = (unsigned)(((size_t)rows * 32 + threads - 1) / threads);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(blocks);
+  cfg.blockDim = dim3(threads);
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t err = cudaSuccess;
+#define RS_CASE(N) \
+  case N: err = cudaLaunchKernelEx(&cfg, rowstats_bf16_kernel<N>, x, eps, stats, rows, cols); break;
+  switch (nch) {
+    RS_CASE(1) RS_CASE(2) RS_CASE(3) RS_CASE(4) RS_CASE(5) RS_CASE(6) RS_CASE(7) RS_CASE(8)
+    default: return cudaErrorInvalidValue;
+  }
+#undef RS_CASE
+  return err;
+}
+
 // fp32 LayerNorm: one warp per row, two passes over global memory.
 __global__ void layernorm_f32_kernel(const float* __restrict__ x, const float* __restrict__ g,
                                      const float* __restrict__ b, float eps, float* __restrict__ y,

@@ -67,7 +67,7 @@ size_t stage_ws_bytes(const vit_config& c, int mb) {
   const size_t act = c.dtype == VIT_BF16 ? 2 : 4;
   const size_t M = (size_t)mb * s.T;
   const size_t wide = 3 * s.H > s.F ? 3 * s.H : s.F;
-  return align_up(M * s.H * act, 256) + align_up(M * wide * act, 256);
+  return align_up(M * s.H * act, 256) + align_up(M * wide * act, 256) + align_up(M * sizeof(float2), 256);
 }
 size_t embed_ws_bytes(const vit_config& c, int mb) {
   const Shape s(c);
@@ -101,11 +101,15 @@ PipeLayout pipe_layout(const vit_config& c, int mb) {
 inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; }
 
 // Converts n fp32 values to the device element type into dst (host staging).
-void convert_matrix(const float* src, void* dst, size_t rows, size_t cols, size_t cols_pad, bool to_bf16) {
+void convert_matrix(const float* src, void* dst, size_t rows, size_t cols, size_t cols_pad, bool to_bf16,
+                    const float* col_scale = nullptr) {
   if (to_bf16) {
     bf16* d = static_cast<bf16*>(dst);
     for (size_t r = 0; r < rows; ++r) {
-      for (size_t c = 0; c < cols; ++c) d[r * cols_pad + c] = __float2bfloat16_rn(src[r * cols + c]);
+      if (col_scale)
+        for (size_t c = 0; c < cols; ++c) d[r * cols_pad + c] = __float2bfloat16_rn(src[r * cols + c] * col_scale[c]);
+      else
+        for (size_t c = 0; c < cols; ++c) d[r * cols_pad + c] = __float2bfloat16_rn(src[r * cols + c]);
       for (size_t c = cols; c < cols_pad; ++c) d[r * cols_pad + c] = __float2bfloat16_rn(0.f);
     }
   } else {
@@ -254,11 +258,11 @@ int vit_create(const vit_config* cfg, const float* host_params, size_t n_params,
   const int L = cfg->layers;
 
   // device blob layout: every tensor 256-byte aligned
-  struct Item { size_t src, rows, cols, cols_pad; bool matrix; size_t dst; };
+  struct Item { size_t src, rows, cols, cols_pad; bool matrix; size_t dst; const float* col_scale; };
   std::vector<Item> items;
   size_t src = 0, dst = 0;
   auto add = [&](size_t rows, size_t cols, size_t cols_pad, bool matrix) {
-    Item it{src, rows, cols, cols_pad, matrix, dst};
+    Item it{src, rows, cols, cols_pad, matrix, dst, nullptr};
     items.push_back(it);
     src += rows * cols;
     dst += align_up(rows * cols_pad * (matrix ? act : 4), 256);
@@ -291,6 +295,28 @@ int vit_create(const vit_config* cfg, const float* host_params, size_t n_params,
   const size_t i_hdw = s.X ? add(s.C, s.H, s.H, true) : 0;
   const size_t i_hdb = s.X ? add(1, s.C, s.C, false) : 0;
   if (src != n_params) return VIT_ERR_INVALID_ARG;
+  // bf16 mode: LayerNorm 1 and 2 are folded into the QKV and fc1 products.  The gain goes into the
+  // weight (wg[n,k] = g[k] w[n,k], rounded to bf16); per layer four derived vectors follow the
+  // parameters: c1[n] = sum_k wg[n,k] and c0[n] = bias[n] + sum_k shift[k] w[n,k] for each of the two.
+  struct Derived { size_t dst, w_item, g_item, b_item, bias_item; };
+  std::vector<Derived> derived;
+  std::vector<size_t> ld(L, 0);
+  if (b16) {
+    for (int l = 0; l < L; ++l) {
+      const size_t b = li[l];
+      items[b + 2].col_scale = host_params + items[b + 0].src;      // Wqkv * ln1.g
+      items[b + 8].col_scale = host_params + items[b + 6].src;      // W1 * ln2.g
+      ld[l] = derived.size();
+      for (int which = 0; which < 2; ++which) {
+        const size_t w = b + (which ? 8 : 2), g = b + (which ? 6 : 0);
+        const size_t n = items[w].rows;
+        for (int v = 0; v < 2; ++v) {                                // c1 then c0
+          derived.push_back(Derived{dst, w, g, g + 1, w + 1});
+          dst += align_up(n * sizeof(float), 256);
+        }
+      }
+    }
+  }
   const size_t blob_bytes = dst;
 
   uint8_t* staging = static_cast<uint8_t*>(malloc(blob_bytes));
@@ -305,7 +331,26 @@ int vit_create(const vit_config* cfg, const float* host_params, size_t n_params,
         for (size_t i = t; i < items.size(); i += nt) {
           const Item& it = items[i];
           convert_matrix(host_params + it.src, staging + it.dst, it.rows, it.cols, it.cols_pad,
-                         it.matrix && b16);
+                         it.matrix && b16, it.col_scale);
+        }
+        for (size_t i = t; i < derived.size(); i += nt) {
+          const Derived& d = derived[i];
+          const Item& w = items[d.w_item];
+          const float* W = host_params + w.src;
+          const float* g = host_params + items[d.g_item].src;
+          const float* sh = host_params + items[d.b_item].src;
+          const float* bias = host_params + items[d.bias_item].src;
+          float* out = reinterpret_cast<float*>(staging + d.dst);
+          const bool is_c1 = (i % 2) == 0;
+          for (size_t n = 0; n < w.rows; ++n) {
+            double acc = is_c1 ? 0.0 : (double)bias[n];
+            for (size_t k = 0; k < w.cols; ++k) {
+              const float wv = W[n * w.cols + k];
+              acc += is_c1 ? (double)__bfloat162float(__float2bfloat16_rn(wv * g[k]))
+                           : (double)sh[k] * (double)__bfloat162float(__float2bfloat16_rn(wv));
+            }
+            out[n] = (float)acc;
+          }
         }
       });
     }
@@ -343,6 +388,11 @@ int vit_create(const vit_config* cfg, const float* host_params, size_t n_params,
     w.ln1_g = fp(b); w.ln1_b = fp(b + 1); w.Wqkv = vp(b + 2); w.bqkv = fp(b + 3);
     w.Wo = vp(b + 4); w.bo = fp(b + 5); w.ln2_g = fp(b + 6); w.ln2_b = fp(b + 7);
     w.W1 = vp(b + 8); w.b1 = fp(b + 9); w.W2 = vp(b + 10); w.b2 = fp(b + 11);
+    w.qkv_c1 = w.qkv_c0 = w.fc1_c1 = w.fc1_c0 = nullptr;
+    if (b16) {
+      auto dp = [&](size_t i) { return reinterpret_cast<const float*>(B + derived[ld[l] + i].dst); };
+      w.qkv_c1 = dp(0); w.qkv_c0 = dp(1); w.fc1_c1 = dp(2); w.fc1_c0 = dp(3);
+    }
   }
   h->lnf_g = fp(i_lnfg); h->lnf_b = fp(i_lnfb); h->head_W = vp(i_hw); h->head_b = fp(i_hb);
   h->head_dist_W = s.X ? vp(i_hdw) : nullptr; h->head_dist_b = s.X ? fp(i_hdb) : nullptr;
@@ -401,20 +451,28 @@ int vit_run_stage(vit_handle* h, int layer_begin, int layer_end, int mb, const v
   }
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const bool b16 = c.dtype == VIT_BF16;
-  uint8_t* y = static_cast<uint8_t*>(ws);                       // [M, H]: LN output, then attention output
+  uint8_t* y = static_cast<uint8_t*>(ws);                       // [M, H]: attention output (fp32 mode: also the LN output)
   uint8_t* wide = y + align_up(tok_bytes, 256);                 // [M, 3H] qkv, later [M, F] MLP hidden
+  const size_t wide_cols = 3 * H > F ? 3 * H : F;
+  float2* stats = reinterpret_cast<float2*>(wide + align_up(M * wide_cols * h->act_bytes, 256));   // [M] LayerNorm statistics
 
   for (int l = layer_begin; l < layer_end; ++l) {
     const LayerWeights& w = h->layers[l];
     const void* x_in = (l == layer_begin) ? in : out;
-    // y = LN1(x)
-    if (b16) VIT_LAUNCH(h, VIT_PROF_LAYERNORM, launch_layernorm_bf16((const bf16*)x_in, w.ln1_g, w.ln1_b, c.ln_eps, (bf16*)y, (int)M, (int)H, s));
-    else VIT_LAUNCH(h, VIT_PROF_LAYERNORM, launch_layernorm_f32((const float*)x_in, w.ln1_g, w.ln1_b, c.ln_eps, (float*)y, (int)M, (int)H, s));
-    // qkv = y Wqkv^T + bqkv
     LinearArgs a{};
-    a.M = (int)M; a.N = (int)(3 * H); a.K = (int)H;
-    a.a = y; a.lda = (int)H; a.w = w.Wqkv; a.ldw = (int)H; a.bias = w.bqkv;
-    a.epilogue = EPI_BIAS; a.out = wide; a.ldo = (int)(3 * H);
+    if (b16) {
+      // LN1 folded into the QKV product: row statistics of x, then qkv = LN1(x) Wqkv^T + bqkv from the raw rows
+      VIT_LAUNCH(h, VIT_PROF_LAYERNORM, launch_rowstats_bf16((const bf16*)x_in, c.ln_eps, stats, (int)M, (int)H, s));
+      a.M = (int)M; a.N = (int)(3 * H); a.K = (int)H;
+      a.a = x_in; a.lda = (int)H; a.w = w.Wqkv; a.ldw = (int)H; a.bias = w.qkv_c0;
+      a.epilogue = EPI_LN_BIAS; a.ln_stats = stats; a.ln_c1 = w.qkv_c1; a.out = wide; a.ldo = (int)(3 * H);
+    } else {
+      // y = LN1(x); qkv = y Wqkv^T + bqkv
+      VIT_LAUNCH(h, VIT_PROF_LAYERNORM, launch_layernorm_f32((const float*)x_in, w.ln1_g, w.ln1_b, c.ln_eps, (float*)y, (int)M, (int)H, s));
+      a.M = (int)M; a.N = (int)(3 * H); a.K = (int)H;
+      a.a = y; a.lda = (int)H; a.w = w.Wqkv; a.ldw = (int)H; a.bias = w.bqkv;
+      a.epilogue = EPI_BIAS; a.out = wide; a.ldo = (int)(3 * H);
+    }
     if ((st = linear(h, VIT_PROF_QKV, a, s)) != VIT_OK) return st;
     // y = attention(qkv)
     if (b16) VIT_LAUNCH(h, VIT_PROF_ATTENTION, launch_attention_bf16((const bf16*)wide, (bf16*)y, mb, h->T, c.heads, h->d, h->dev_status, s));
@@ -425,14 +483,19 @@ int vit_run_stage(vit_handle* h, int layer_begin, int layer_end, int mb, const v
     a.a = y; a.lda = (int)H; a.w = w.Wo; a.ldw = (int)H; a.bias = w.bo;
     a.epilogue = EPI_BIAS_RESIDUAL; a.residual = x_in; a.out = out; a.ldo = (int)H;
     if ((st = linear(h, VIT_PROF_OUTPROJ, a, s)) != VIT_OK) return st;
-    // y = LN2(x)
-    if (b16) VIT_LAUNCH(h, VIT_PROF_LAYERNORM, launch_layernorm_bf16((const bf16*)out, w.ln2_g, w.ln2_b, c.ln_eps, (bf16*)y, (int)M, (int)H, s));
-    else VIT_LAUNCH(h, VIT_PROF_LAYERNORM, launch_layernorm_f32((const float*)out, w.ln2_g, w.ln2_b, c.ln_eps, (float*)y, (int)M, (int)H, s));
-    // u = gelu(y W1^T + b1)
+    // u = gelu(LN2(x) W1^T + b1)
     a = LinearArgs{};
-    a.M = (int)M; a.N = (int)F; a.K = (int)H;
-    a.a = y; a.lda = (int)H; a.w = w.W1; a.ldw = (int)H; a.bias = w.b1;
-    a.epilogue = EPI_BIAS_GELU; a.out = wide; a.ldo = (int)F;
+    if (b16) {
+      VIT_LAUNCH(h, VIT_PROF_LAYERNORM, launch_rowstats_bf16((const bf16*)out, c.ln_eps, stats, (int)M, (int)H, s));
+      a.M = (int)M; a.N = (int)F; a.K = (int)H;
+      a.a = out; a.lda = (int)H; a.w = w.W1; a.ldw = (int)H; a.bias = w.fc1_c0;
+      a.epilogue = EPI_LN_BIAS_GELU; a.ln_stats = stats; a.ln_c1 = w.fc1_c1; a.out = wide; a.ldo = (int)F;
+    } else {
+      VIT_LAUNCH(h, VIT_PROF_LAYERNORM, launch_layernorm_f32((const float*)out, w.ln2_g, w.ln2_b, c.ln_eps, (float*)y, (int)M, (int)H, s));
+      a.M = (int)M; a.N = (int)F; a.K = (int)H;
+      a.a = y; a.lda = (int)H; a.w = w.W1; a.ldw = (int)H; a.bias = w.b1;
+      a.epilogue = EPI_BIAS_GELU; a.out = wide; a.ldo = (int)F;
+    }
     if ((st = linear(h, VIT_PROF_FC1, a, s)) != VIT_OK) return st;
     // x = x + u W2^T + b2
     a = LinearArgs{};
@@ -595,6 +658,29 @@ int vit_op_linear_tiled(vit_handle* h, int dtype, int M, int N, int K, const voi
   } else {
     return VIT_ERR_INVALID_ARG;
   }
+  return VIT_OK;
+}
+
+int vit_op_rowstats(vit_handle* h, int rows, int cols, const void* x, float eps, float* stats, void* stream) {
+  if (!h || !x || !stats || rows < 0 || cols < 1 || cols % 8 || !on_own_device(h)) return VIT_ERR_INVALID_ARG;
+  if (misaligned(x) || misaligned(stats)) return VIT_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  VIT_LAUNCH(h, VIT_PROF_LAYERNORM, launch_rowstats_bf16((const bf16*)x, eps, reinterpret_cast<float2*>(stats), rows, cols, s));
+  return VIT_OK;
+}
+
+int vit_op_linear_ln(vit_handle* h, int M, int N, int K, const void* a, const float* stats, const void* wg,
+                     const float* c1, const float* c0, int gelu, void* out, int tiling, void* stream) {
+  if (!h || !a || !stats || !wg || !c1 || !c0 || !out || M < 0 || N < 1 || K < 1 || !on_own_device(h)) return VIT_ERR_INVALID_ARG;
+  if (K % 8 || N % 8 || tiling < VIT_TILING_AUTO || tiling > VIT_TILING_PAIR_256x256) return VIT_ERR_INVALID_ARG;
+  if (misaligned(a) || misaligned(stats) || misaligned(wg) || misaligned(c1) || misaligned(c0) || misaligned(out))
+    return VIT_ERR_INVALID_ARG;
+  LinearArgs p{};
+  p.M = M; p.N = N; p.K = K; p.a = a; p.lda = K; p.w = wg; p.ldw = K; p.bias = c0;
+  p.epilogue = gelu ? EPI_LN_BIAS_GELU : EPI_LN_BIAS;
+  p.ln_stats = reinterpret_cast<const float2*>(stats); p.ln_c1 = c1; p.out = out; p.ldo = N; p.tiling = tiling;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  VIT_LAUNCH(h, VIT_PROF_OP, launch_linear_tc(p, h->dev_status, s));
   return VIT_OK;
 }
 

@@ -19,8 +19,14 @@ enum Epilogue : int {
   EPI_BIAS = 0,          // out = acc + bias
   EPI_BIAS_GELU = 1,     // out = gelu(acc + bias), erf form
   EPI_BIAS_RESIDUAL = 2, // out = acc + bias + residual[row, col]
-  EPI_BIAS_POS = 3       // patch embed: row r of the GEMM is patch r % n_patches of image r / n_patches;
+  EPI_BIAS_POS = 3,      // patch embed: row r of the GEMM is patch r % n_patches of image r / n_patches;
                          // out[image*T + t0 + patch, col] = acc + bias + pos[t0 + patch, col], T = t0 + n_patches
+  // LayerNorm of the input rows folded into the product (bf16 tensor-core kernel only): with the
+  // gain folded into the weight, wg[n,k] = g[k] w[n,k], the kernel multiplies the raw rows and applies
+  //   out[m,n] = rstd[m] (acc[m,n] - mean[m] c1[n]) + c0[n],  c1[n] = sum_k wg[n,k],  c0[n] = sum_k b[k] w[n,k] + bias[n]
+  // which equals LN(a)[m,:] . w[n,:] + bias[n] without a normalised copy of a ever being written.
+  EPI_LN_BIAS = 4,
+  EPI_LN_BIAS_GELU = 5
 };
 
 struct LinearArgs {
@@ -33,6 +39,8 @@ struct LinearArgs {
   int epilogue;
   const void* residual;   // EPI_BIAS_RESIDUAL: [M, N] stride ldo; may alias out
   const float* pos;       // EPI_BIAS_POS: [T, N] fp32
+  const float2* ln_stats; // EPI_LN_*: [M] (mean, 1/sqrt(var + eps)) of the rows of a
+  const float* ln_c1;     // EPI_LN_*: [N] row sums of the gain-folded weight; bias holds c0
   int n_patches;          // EPI_BIAS_POS
   int first_patch_token;  // EPI_BIAS_POS: t0, the number of special tokens before the patches
   void* out;              // activation type, row stride ldo
@@ -45,7 +53,8 @@ enum Tiling : int { TILING_AUTO = 0, TILING_128x128 = 1, TILING_128x256 = 2, TIL
 
 struct LayerWeights {
   const float *ln1_g, *ln1_b, *bqkv, *bo, *ln2_g, *ln2_b, *b1, *b2;
-  const void *Wqkv, *Wo, *W1, *W2;   // activation type, [out, in]
+  const void *Wqkv, *Wo, *W1, *W2;   // activation type, [out, in]; bf16 mode: Wqkv and W1 carry the LayerNorm gain
+  const float *qkv_c1, *qkv_c0, *fc1_c1, *fc1_c0;   // bf16 mode: the folded LayerNorm's column vectors (see EPI_LN_BIAS)
 };
 
 struct ProfRecord { cudaEvent_t begin, end; int cls; };
@@ -74,6 +83,8 @@ struct Handle {
 cudaError_t launch_layernorm_bf16(const bf16* x, const float* g, const float* b, float eps,
                                   bf16* y, int rows, int cols, cudaStream_t s);
 cudaError_t launch_linear_tc(const LinearArgs& a, int* dev_status, cudaStream_t s);   // tcgen05 GEMM
+// per-row LayerNorm statistics: stats[r] = (mean, 1 / sqrt(biased variance + eps)) of x[r, :]
+cudaError_t launch_rowstats_bf16(const bf16* x, float eps, float2* stats, int rows, int cols, cudaStream_t s);
 // attention: the tcgen05 kernel where it supports the shape, else the warp-level mma kernel
 cudaError_t launch_attention_bf16(const bf16* qkv, bf16* out, int images, int T, int heads, int d,
                                   int* dev_status, cudaStream_t s);

@@ -58,14 +58,15 @@ def test_workspace_sizes(L):
     shape = vitgen.preset("huge14")
     cfg = vit.make_config(shape, vit.VIT_BF16, 128)
     M = 128 * 257
-    stage = M * 1280 * 2 + M * 5120 * 2
+    stage = M * 1280 * 2 + M * 5120 * 2 + M * 8      # attention output, QKV / MLP hidden, LayerNorm statistics
     assert vit.vit_workspace_bytes(cfg, 128) >= stage
     assert vit.vit_workspace_bytes(cfg, 128) < stage + 4096
     assert vit.vit_workspace_bytes(cfg, 0) == 0
     pipe = vit.vit_pipeline_workspace_bytes(cfg, 8)
     assert pipe >= vit.vit_workspace_bytes(cfg, 8) + 8 * 3 * 224 * 224 * 4 + 8 * 257 * 1280 * 2
     cfg32 = vit.make_config(shape, vit.VIT_FP32, 128)
-    assert vit.vit_workspace_bytes(cfg32, 4) >= 2 * (vit.vit_workspace_bytes(cfg, 4) - 512)
+    # twice the activation buffers of the bf16 mode (the statistics buffer has the same size in both)
+    assert vit.vit_workspace_bytes(cfg32, 4) >= 2 * (vit.vit_workspace_bytes(cfg, 4) - 768 - 4 * 257 * 8)
 
 
 def test_status_strings(L):

@@ -52,6 +52,59 @@ def test_layernorm_bf16(ctx, rows, cols):
     assert np.abs(got - want).max() <= BF16_EPS * np.abs(want).max() + 1e-5
 
 
+@pytest.mark.parametrize("rows,cols", [(1, 192), (5, 768), (1031, 1280), (33, 64)])
+def test_rowstats_bf16(ctx, rows, cols):
+    vit, m = ctx
+    rng = np.random.default_rng(rows + 3 * cols)
+    x, xr = _bf16(rng.normal(0.7, 1.5, size=(rows, cols)))
+    stats = torch.full((rows, 2), float("nan"), dtype=torch.float32, device="cuda")
+    vit.vit_op_rowstats(m.h, rows, cols, x.data_ptr(), 1e-6, stats.data_ptr())
+    torch.cuda.synchronize()
+    got = stats.cpu().numpy()
+    mean = xr.mean(-1)
+    rstd = 1.0 / np.sqrt(((xr - mean[:, None]) ** 2).mean(-1) + 1e-6)     # the two quantities of the oracle's layernorm
+    np.testing.assert_allclose(got[:, 0], mean, rtol=0, atol=2e-6 * np.abs(xr).max())
+    np.testing.assert_allclose(got[:, 1], rstd, rtol=2e-6)
+
+
+# LayerNorm folded into the product: compared with the oracle's layernorm -> linear (-> gelu) on
+# the same rows, every tiling; the test folds gain and shift into the operands the way vit_create does
+@pytest.mark.parametrize("M,N,K", [(300, 1000 // 8 * 8, 328), (257 * 16, 3840, 1280), (257 * 16, 5120, 1280)])
+@pytest.mark.parametrize("tiling", [1, 2, 3])
+@pytest.mark.parametrize("gelu", [0, 1])
+def test_linear_with_folded_layernorm(ctx, M, N, K, gelu, tiling):
+    vit, m = ctx
+    rng = np.random.default_rng(M + N + K + gelu)
+    x, xr = _bf16(rng.normal(0.3, 2.0, size=(M, K)))
+    g = 1 + 0.2 * rng.normal(size=K)
+    b = 0.3 * rng.normal(size=K)
+    w = rng.normal(size=(N, K)) / np.sqrt(K)
+    wq = torch.from_numpy(w.astype(np.float32)).to(torch.bfloat16).float().numpy().astype(np.float64)   # weight as the model holds it
+    bias = rng.normal(size=N)
+    wg, wgr = _bf16(wq * g[None, :])
+    c1, _ = _f32(wgr.sum(-1))
+    c0, _ = _f32(bias + wq @ b)
+    stats = torch.empty((M, 2), dtype=torch.float32, device="cuda")
+    out = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    vit.vit_op_rowstats(m.h, M, K, x.data_ptr(), 1e-6, stats.data_ptr())
+    vit.vit_op_linear_ln(m.h, M, N, K, x.data_ptr(), stats.data_ptr(), wg.data_ptr(), c1.data_ptr(), c0.data_ptr(),
+                         gelu, out.data_ptr(), tiling)
+    m.check()
+    want = O.linear(O.layernorm(xr, g, b, 1e-6), wq, bias)
+    if gelu:
+        want = O.gelu(want)
+    got = out.float().cpu().numpy()
+    assert np.isfinite(got).all()
+    err = np.abs(got - want)
+    # output rounding to bf16; the bf16 rounding of gain * weight (uniform within 2^-9 relative per
+    # term, K random terms: standard deviation 2^-9 / sqrt(3) of the outputs' scale, bounded here at
+    # seven standard deviations); fp32 accumulation
+    scale = np.sqrt((want ** 2).mean())
+    tol = BF16_EPS * np.abs(want) + 7 * 2.0 ** -9 / np.sqrt(3) * scale + 4e-6 * np.sqrt(K)
+    bad = err > tol
+    assert not bad.any(), (int(bad.sum()), float(err.max()), np.argwhere(bad)[:5].tolist())
+
+
 @pytest.mark.parametrize("rows,cols", [(3, 192), (200, 1280), (7, 100)])
 def test_layernorm_fp32(ctx, rows, cols):
     vit, m = ctx

@@ -1,5 +1,5 @@
 """Per-layer stage times measured on this GPU (the analogue of the paper's per-layer timing
-figure) fed to the pipeline partitioner:  python -m paper_2110_14895_b200.partition_demo
+figure) fed to the pipeline partitioner:  python partition_demo.py
 The devices are this GPU at the given relative speeds; links carry `--gbs` GB/s."""
 import argparse
 import os
@@ -8,7 +8,7 @@ import sys
 import numpy as np
 import torch
 
-sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
 import vitgen  # noqa: E402
 import paper_2110_14895_b200 as vit  # noqa: E402
 

@@ -1,12 +1,16 @@
 """Runs one kernel of the library a few times on random device data, for ncu captures and
-quick timing:  python -m paper_2110_14895_b200.profile_ops --op linear --M 32896 --N 5120 --K 1280 --epilogue 1
+quick timing:  python profile_ops.py --op linear --M 32896 --N 5120 --K 1280 --epilogue 1
 Prints the mean CUDA-event time per launch."""
 import argparse
+
+import os
+import sys
 
 import numpy as np
 import torch
 
-import paper_2110_14895_b200 as vit
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
+import paper_2110_14895_b200 as vit  # noqa: E402
 
 
 class _Shape:
@@ -15,7 +19,7 @@ class _Shape:
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--op", required=True, choices=["linear", "attention", "layernorm"])
+    ap.add_argument("--op", required=True, choices=["linear", "linear_ln", "attention", "layernorm", "rowstats"])
     ap.add_argument("--M", type=int, default=32896)
     ap.add_argument("--N", type=int, default=1280)
     ap.add_argument("--K", type=int, default=1280)
@@ -40,6 +44,25 @@ def main():
                                         a.epilogue, res, out.data_ptr())
         work = 2.0 * a.M * a.N * a.K
         unit = "TFLOP/s"
+    elif a.op == "linear_ln":
+        # the QKV / fc1 product with the LayerNorm folded in (epilogue 0 = plain, 1 = GELU)
+        x = torch.randn(a.M, a.K, device="cuda").to(bf)
+        w = (torch.randn(a.N, a.K, device="cuda") / a.K ** 0.5).to(bf)
+        c1 = w.float().sum(-1).contiguous()
+        c0 = torch.randn(a.N, device="cuda")
+        stats = torch.empty(a.M, 2, device="cuda")
+        out = torch.empty(a.M, a.N, device="cuda", dtype=bf)
+        vit.vit_op_rowstats(h, a.M, a.K, x.data_ptr(), 1e-6, stats.data_ptr())
+        run = lambda: vit.vit_op_linear_ln(h, a.M, a.N, a.K, x.data_ptr(), stats.data_ptr(), w.data_ptr(), c1.data_ptr(),
+                                           c0.data_ptr(), a.epilogue, out.data_ptr())
+        work = 2.0 * a.M * a.N * a.K
+        unit = "TFLOP/s"
+    elif a.op == "rowstats":
+        x = torch.randn(a.M, a.N, device="cuda").to(bf)
+        stats = torch.empty(a.M, 2, device="cuda")
+        run = lambda: vit.vit_op_rowstats(h, a.M, a.N, x.data_ptr(), 1e-6, stats.data_ptr())
+        work = (a.M * a.N * 2 + a.M * 8) / 1e-3     # bytes, scaled so the print below reads GB/s
+        unit = "GB/s"
     elif a.op == "attention":
         H = a.heads * a.d
         qkv = torch.randn(a.images * a.T, 3 * H, device="cuda").to(bf)

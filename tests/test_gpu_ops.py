@@ -90,19 +90,20 @@ def test_linear_with_folded_layernorm(ctx, M, N, K, gelu, tiling):
     vit.vit_op_linear_ln(m.h, M, N, K, x.data_ptr(), stats.data_ptr(), wg.data_ptr(), c1.data_ptr(), c0.data_ptr(),
                          gelu, out.data_ptr(), tiling)
     m.check()
-    want = O.linear(O.layernorm(xr, g, b, 1e-6), wq, bias)
-    if gelu:
-        want = O.gelu(want)
+    pre = O.linear(O.layernorm(xr, g, b, 1e-6), wq, bias)
+    want = O.gelu(pre) if gelu else pre
     got = out.float().cpu().numpy()
     assert np.isfinite(got).all()
     err = np.abs(got - want)
     # output rounding to bf16; the bf16 rounding of gain * weight (uniform within 2^-9 relative per
     # term, K random terms: standard deviation 2^-9 / sqrt(3) of the outputs' scale, bounded here at
     # seven standard deviations); fp32 accumulation
-    scale = np.sqrt((want ** 2).mean())
-    tol = BF16_EPS * np.abs(want) + 7 * 2.0 ** -9 / np.sqrt(3) * scale + 4e-6 * np.sqrt(K)
+    scale = np.sqrt((pre ** 2).mean())               # of the product before the activation (|gelu'| <= 1.13)
+    tol = BF16_EPS * np.abs(want) + 1.13 * 7 * 2.0 ** -9 / np.sqrt(3) * scale + 4e-6 * np.sqrt(K)
     bad = err > tol
-    assert not bad.any(), (int(bad.sum()), float(err.max()), np.argwhere(bad)[:5].tolist())
+    where = np.argwhere(bad)[:3]
+    assert not bad.any(), (int(bad.sum()), float(err.max()), where.tolist(),
+                           [(float(want[i, j]), float(got[i, j]), float(pre[i, j])) for i, j in where])
 
 
 @pytest.mark.parametrize("rows,cols", [(3, 192), (200, 1280), (7, 100)])

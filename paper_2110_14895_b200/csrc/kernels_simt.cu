@@ -141,31 +141,32 @@ rowstats_bf16_kernel(const bf16* __restrict__ x, float eps, float2* __restrict__
     const int idx = lane + 32 * i;
     u[i] = idx < nvec ? __ldg(xr + idx) : make_uint4(0, 0, 0, 0);
   }
-  float v[NCH][8];
-  float sum = 0.f;
+  // unpacked pairs (low half by shift, high half by mask); sums on packed two-wide fp32 instructions
+  float2 v[NCH][4];
+  float2 sum2 = make_float2(0.f, 0.f);
 #pragma unroll
   for (int i = 0; i < NCH; ++i) {
     const uint32_t w[4] = {u[i].x, u[i].y, u[i].z, u[i].w};
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      v[i][2 * e] = __uint_as_float(w[e] << 16);
-      v[i][2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
-      sum += v[i][2 * e] + v[i][2 * e + 1];
+      v[i][e] = make_float2(__uint_as_float(w[e] << 16), __uint_as_float(w[e] & 0xffff0000u));
+      sum2 = __fadd2_rn(sum2, v[i][e]);          // padded chunks are zero
     }
   }
-  const float mean = warp_sum(sum) / (float)cols;
-  float sq = 0.f;
+  const float mean = warp_sum(sum2.x + sum2.y) / (float)cols;
+  const float2 nmean = make_float2(-mean, -mean);
+  float2 sq2 = make_float2(0.f, 0.f);
 #pragma unroll
   for (int i = 0; i < NCH; ++i) {
     if (lane + 32 * i < nvec) {
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const float c = v[i][e] - mean;
-        sq = fmaf(c, c, sq);
+      for (int e = 0; e < 4; ++e) {
+        const float2 c = __fadd2_rn(v[i][e], nmean);
+        sq2 = __ffma2_rn(c, c, sq2);
       }
     }
   }
-  const float rstd = 1.0f / sqrtf(warp_sum(sq) / (float)cols + eps);
+  const float rstd = 1.0f / sqrtf(warp_sum(sq2.x + sq2.y) / (float)cols + eps);
   if (lane == 0) stats[row] = make_float2(mean, rstd);
 }
 

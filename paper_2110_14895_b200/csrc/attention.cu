@@ -200,9 +200,9 @@ cudaError_t launch_d(const bf16* qkv, bf16* out, int images, int T, int heads, c
 }  // namespace
 
 cudaError_t launch_attention_bf16(const bf16* qkv, bf16* out, int images, int T, int heads, int d,
-                                  int* dev_status, cudaStream_t s) {
+                                  int* dev_status, cudaStream_t s, TensorMapCache* cache) {
   if (images <= 0) return cudaSuccess;
-  if (attention_tc_supported(T, d)) return launch_attention_tc(qkv, out, images, T, heads, d, dev_status, s);
+  if (attention_tc_supported(T, d)) return launch_attention_tc(qkv, out, images, T, heads, d, dev_status, s, cache);
   switch (d) {
     case 16: return launch_d<16>(qkv, out, images, T, heads, s);
     case 32: return launch_d<32>(qkv, out, images, T, heads, s);

@@ -625,8 +625,16 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
 
-bool encode_map(CUtensorMap* tm, const void* base, size_t rows, size_t cols, int box_cols, int box_rows,
-                CUtensorMapSwizzle sw) {
+bool encode_map_raw(CUtensorMap* tm, const void* base, size_t rows, size_t cols, int box_cols, int box_rows,
+                    CUtensorMapSwizzle sw);
+bool encode_map(TensorMapCache* cache, CUtensorMap* tm, const void* base, size_t rows, size_t cols, int box_cols,
+                int box_rows, CUtensorMapSwizzle sw) {
+  const TensorMapKey key{base, (uint64_t)rows, (uint64_t)cols, (uint64_t)cols, (uint32_t)box_rows, (uint32_t)box_cols,
+                         (uint32_t)sw + 1000u};
+  return TensorMapCache::get(cache, key, tm, [&](CUtensorMap* out) { return encode_map_raw(out, base, rows, cols, box_cols, box_rows, sw); });
+}
+bool encode_map_raw(CUtensorMap* tm, const void* base, size_t rows, size_t cols, int box_cols, int box_rows,
+                    CUtensorMapSwizzle sw) {
   const cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   const cuuint64_t gstride[1] = {(cuuint64_t)cols * 2};
   const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
@@ -638,7 +646,7 @@ bool encode_map(CUtensorMap* tm, const void* base, size_t rows, size_t cols, int
 
 template <int D, int NKP>
 cudaError_t launch_variant(const bf16* qkv, bf16* out, int images, int T, int heads, int* dev_status,
-                           cudaStream_t s) {
+                           cudaStream_t s, TensorMapCache* cache) {
   using L = Smem<D, NKP>;
   if (!g_encode) {
     void* fn = nullptr;
@@ -656,13 +664,13 @@ cudaError_t launch_variant(const bf16* qkv, bf16* out, int images, int T, int he
   const size_t rows = (size_t)images * T, cols = (size_t)3 * heads * D;
   const CUtensorMapSwizzle s128 = CU_TENSOR_MAP_SWIZZLE_128B, s32 = CU_TENSOR_MAP_SWIZZLE_32B;
   AttnMaps m;
-  if (!encode_map(&m.q64, qkv, rows, cols, 64, QT, s128)) return cudaErrorInvalidValue;
-  if (!encode_map(&m.k64m, qkv, rows, cols, 64, NKP, s128)) return cudaErrorInvalidValue;
-  if (!encode_map(&m.k64x, qkv, rows, cols, 64, 16, s128)) return cudaErrorInvalidValue;
+  if (!encode_map(cache, &m.q64, qkv, rows, cols, 64, QT, s128)) return cudaErrorInvalidValue;
+  if (!encode_map(cache, &m.k64m, qkv, rows, cols, 64, NKP, s128)) return cudaErrorInvalidValue;
+  if (!encode_map(cache, &m.k64x, qkv, rows, cols, 64, 16, s128)) return cudaErrorInvalidValue;
   if (D > 64) {
-    if (!encode_map(&m.q16, qkv, rows, cols, 16, QT, s32)) return cudaErrorInvalidValue;
-    if (!encode_map(&m.k16m, qkv, rows, cols, 16, NKP, s32)) return cudaErrorInvalidValue;
-    if (!encode_map(&m.k16x, qkv, rows, cols, 16, 16, s32)) return cudaErrorInvalidValue;
+    if (!encode_map(cache, &m.q16, qkv, rows, cols, 16, QT, s32)) return cudaErrorInvalidValue;
+    if (!encode_map(cache, &m.k16m, qkv, rows, cols, 16, NKP, s32)) return cudaErrorInvalidValue;
+    if (!encode_map(cache, &m.k16x, qkv, rows, cols, 16, 16, s32)) return cudaErrorInvalidValue;
   } else {
     m.q16 = m.q64;
     m.k16m = m.k64m;
@@ -690,14 +698,14 @@ bool attention_tc_supported(int T, int d) {
 }
 
 cudaError_t launch_attention_tc(const bf16* qkv, bf16* out, int images, int T, int heads, int d,
-                                int* dev_status, cudaStream_t s) {
+                                int* dev_status, cudaStream_t s, TensorMapCache* cache) {
   if (images <= 0) return cudaSuccess;
   if (!attention_tc_supported(T, d)) return cudaErrorInvalidValue;
   const bool wide = T > 208;
-  if (d == 64) return wide ? launch_variant<64, 256>(qkv, out, images, T, heads, dev_status, s)
-                           : launch_variant<64, 208>(qkv, out, images, T, heads, dev_status, s);
-  return wide ? launch_variant<80, 256>(qkv, out, images, T, heads, dev_status, s)
-              : launch_variant<80, 208>(qkv, out, images, T, heads, dev_status, s);
+  if (d == 64) return wide ? launch_variant<64, 256>(qkv, out, images, T, heads, dev_status, s, cache)
+                           : launch_variant<64, 208>(qkv, out, images, T, heads, dev_status, s, cache);
+  return wide ? launch_variant<80, 256>(qkv, out, images, T, heads, dev_status, s, cache)
+              : launch_variant<80, 208>(qkv, out, images, T, heads, dev_status, s, cache);
 }
 
 }  // namespace vit

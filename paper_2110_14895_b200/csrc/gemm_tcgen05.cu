@@ -30,6 +30,7 @@ constexpr int BK = 64;        // 64 bf16 = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;
 constexpr int NUM_EPI_WARPS = 8;
 constexpr int NUM_THREADS = (2 + NUM_EPI_WARPS) * 32;
+constexpr long long DRAIN_LIMIT_CYCLES = 1ll << 24;   // teardown after a failed wait: ~10 ms per barrier
 
 template <int BN, int CTAS> struct Cfg {
   static constexpr int B_ROWS = BN / CTAS;                 // rows of the w tile this CTA loads
@@ -122,7 +123,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
   uint64_t* tfull_bar = bars + 2 * C::STAGES;      // [2]
   uint64_t* tempty_bar = bars + 2 * C::STAGES + 2; // [2]
   uint64_t* res_bar = bars + 2 * C::STAGES + 4;    // [NUM_EPI_WARPS] residual tile landed
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * C::STAGES + 4 + NUM_EPI_WARPS);
+  uint64_t* drain_bar = bars + 2 * C::STAGES + 4 + NUM_EPI_WARPS;   // teardown after a failed wait
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * C::STAGES + 5 + NUM_EPI_WARPS);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -143,6 +145,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       mbar_init(smem_u32(&tempty_bar[i]), NUM_EPI_WARPS * CTAS);
     }
     for (int i = 0; i < NUM_EPI_WARPS; ++i) mbar_init(smem_u32(&res_bar[i]), 1);
+    mbar_init(smem_u32(drain_bar), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_a)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tm_w)) : "memory");
@@ -167,12 +170,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
+      long long fills = 0;                         // stages filled so far (this CTA's share)
       bool ok = true;
       for (int tile = unit; tile < total_tiles && ok; tile += num_units) {
         const int m0 = (tile / p.tiles_n) * (BM * CTAS) + (int)rank * BM;
         const int n0 = (tile % p.tiles_n) * BN + (int)rank * C::B_ROWS;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1, abort_flag)) { ok = false; break; }
+          ++fills;
           const uint32_t fb = smem_u32(&full_bar[stage]);
           const uint32_t sa = smem_u32(tiles + stage * C::STAGE_BYTES);
           if (CTAS == 2) {
@@ -187,6 +192,20 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
             tma_load_2d(sa + C::A_BYTES, &tm_w, kb * BK, n0, fb);
           }
           if (++stage == C::STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+      if (*abort_flag) {
+        // A wait gave up somewhere in this CTA (or its partner).  The copies of the last STAGES
+        // fills may still be in flight: wait, bounded, until each of those stages has received its
+        // bytes, so that nothing lands in shared memory after the CTA has left.  In a pair the
+        // barriers live in the even CTA and count both CTAs' bytes; the odd CTA is kept alive by
+        // the cluster barrier of the teardown until the even one is through here.
+        if (rank == 0) {
+          volatile int never = 0;
+          const long long first = fills > C::STAGES ? fills - C::STAGES : 0;
+          for (long long f = first; f < fills; ++f)
+            mbar_wait_limit(smem_u32(&full_bar[(int)(f % C::STAGES)]), (uint32_t)((f / C::STAGES) & 1), &never,
+                            DRAIN_LIMIT_CYCLES);
         }
       }
     }
@@ -228,6 +247,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         if (CTAS == 2) umma_commit_pair(smem_u32(&tfull_bar[buf]));   // accumulator complete
         else umma_commit(smem_u32(&tfull_bar[buf]));
         if (++buf == 2) { buf = 0; aphase ^= 1; }
+      }
+      if (*abort_flag) {
+        // products issued so far retire before tensor memory is freed
+        volatile int never = 0;
+        umma_commit(smem_u32(drain_bar));
+        mbar_wait_limit(smem_u32(drain_bar), 0, &never, DRAIN_LIMIT_CYCLES);
       }
     }
   } else {
@@ -403,7 +428,10 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
 
   // ------------------------------------------------------------------ teardown
   __syncwarp();
-  if (*abort_flag) __nanosleep(200000);   // let copies and MMAs in flight land before leaving
+  if (CTAS == 2 && *abort_flag) {
+    // tell the partner, which may be in a wait of its own that nothing will satisfy any more
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(map_to_cta(smem_u32(const_cast<int*>(abort_flag)), rank ^ 1u)), "r"(1) : "memory");
+  }
   tc_fence_before();
   __syncthreads();
   if (CTAS == 2) cluster_sync();          // neither CTA leaves while the other may still touch it
@@ -423,7 +451,12 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
 
-bool encode_2d_bf16(CUtensorMap* tm, const void* base, int rows, int cols, int ld, int box_rows) {
+bool encode_2d_bf16_raw(CUtensorMap* tm, const void* base, int rows, int cols, int ld, int box_rows);
+bool encode_2d_bf16(TensorMapCache* cache, CUtensorMap* tm, const void* base, int rows, int cols, int ld, int box_rows) {
+  const TensorMapKey key{base, (uint64_t)rows, (uint64_t)cols, (uint64_t)ld, (uint32_t)box_rows, (uint32_t)BK, 128u};
+  return TensorMapCache::get(cache, key, tm, [&](CUtensorMap* out) { return encode_2d_bf16_raw(out, base, rows, cols, ld, box_rows); });
+}
+bool encode_2d_bf16_raw(CUtensorMap* tm, const void* base, int rows, int cols, int ld, int box_rows) {
   if (base == nullptr) return false;
   const cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   const cuuint64_t gstride[1] = {(cuuint64_t)ld * 2};
@@ -530,7 +563,7 @@ int current_device_sm_count() {
   return n;
 }
 
-cudaError_t launch_linear_tc(const LinearArgs& a, int* dev_status, cudaStream_t s) {
+cudaError_t launch_linear_tc(const LinearArgs& a, int* dev_status, cudaStream_t s, TensorMapCache* cache) {
   if (a.M <= 0 || a.N <= 0) return cudaSuccess;
   if (!g_encode) return cudaErrorNotReady;
   if (a.K % 8 || a.N % 8 || a.lda % 8 || a.ldw % 8 || a.ldo % 8 || a.K <= 0) return cudaErrorInvalidValue;
@@ -579,12 +612,12 @@ cudaError_t launch_linear_tc(const LinearArgs& a, int* dev_status, cudaStream_t 
   p.tiles_n = (a.N + bn - 1) / bn;
   p.dev_status = dev_status;
   Maps m;
-  if (!encode_2d_bf16(&m.a, a.a, a.M, a.K, a.lda, BM)) return cudaErrorInvalidValue;
-  if (!encode_2d_bf16(&m.w, a.w, a.N, a.K, a.ldw, pair ? bn / 2 : bn)) return cudaErrorInvalidValue;
+  if (!encode_2d_bf16(cache, &m.a, a.a, a.M, a.K, a.lda, BM)) return cudaErrorInvalidValue;
+  if (!encode_2d_bf16(cache, &m.w, a.w, a.N, a.K, a.ldw, pair ? bn / 2 : bn)) return cudaErrorInvalidValue;
   // output (and residual) tiles move as 32-row x 64-column boxes through the epilogue's staging
-  if (!encode_2d_bf16(&m.out, a.out, a.M, a.N, a.ldo, 32)) return cudaErrorInvalidValue;
+  if (!encode_2d_bf16(cache, &m.out, a.out, a.M, a.N, a.ldo, 32)) return cudaErrorInvalidValue;
   if (a.epilogue == EPI_BIAS_RESIDUAL) {
-    if (!encode_2d_bf16(&m.res, a.residual, a.M, a.N, a.ldo, 32)) return cudaErrorInvalidValue;
+    if (!encode_2d_bf16(cache, &m.res, a.residual, a.M, a.N, a.ldo, 32)) return cudaErrorInvalidValue;
   } else {
     m.res = m.out;
   }

@@ -145,7 +145,7 @@ struct ProfScope {
   } while (0)
 
 int linear(Handle* h, int cls, const LinearArgs& a, cudaStream_t s) {
-  if (h->cfg.dtype == VIT_BF16) VIT_LAUNCH(h, cls, launch_linear_tc(a, h->dev_status, s));
+  if (h->cfg.dtype == VIT_BF16) VIT_LAUNCH(h, cls, launch_linear_tc(a, h->dev_status, s, &h->tmaps));
   else VIT_LAUNCH(h, cls, launch_linear_f32(a, s));
   return VIT_OK;
 }
@@ -475,7 +475,7 @@ int vit_run_stage(vit_handle* h, int layer_begin, int layer_end, int mb, const v
     }
     if ((st = linear(h, VIT_PROF_QKV, a, s)) != VIT_OK) return st;
     // y = attention(qkv)
-    if (b16) VIT_LAUNCH(h, VIT_PROF_ATTENTION, launch_attention_bf16((const bf16*)wide, (bf16*)y, mb, h->T, c.heads, h->d, h->dev_status, s));
+    if (b16) VIT_LAUNCH(h, VIT_PROF_ATTENTION, launch_attention_bf16((const bf16*)wide, (bf16*)y, mb, h->T, c.heads, h->d, h->dev_status, s, &h->tmaps));
     else VIT_LAUNCH(h, VIT_PROF_ATTENTION, launch_attention_f32((const float*)wide, (float*)y, mb, h->T, c.heads, h->d, s));
     // x = x + y Wo^T + bo
     a = LinearArgs{};
@@ -652,7 +652,7 @@ int vit_op_linear_tiled(vit_handle* h, int dtype, int M, int N, int K, const voi
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (dtype == VIT_BF16) {
     if (K % 8 || N % 8) return VIT_ERR_INVALID_ARG;
-    VIT_LAUNCH(h, VIT_PROF_OP, launch_linear_tc(p, h->dev_status, s));
+    VIT_LAUNCH(h, VIT_PROF_OP, launch_linear_tc(p, h->dev_status, s, &h->tmaps));
   } else if (dtype == VIT_FP32) {
     VIT_LAUNCH(h, VIT_PROF_OP, launch_linear_f32(p, s));
   } else {
@@ -680,7 +680,7 @@ int vit_op_linear_ln(vit_handle* h, int M, int N, int K, const void* a, const fl
   p.epilogue = gelu ? EPI_LN_BIAS_GELU : EPI_LN_BIAS;
   p.ln_stats = reinterpret_cast<const float2*>(stats); p.ln_c1 = c1; p.out = out; p.ldo = N; p.tiling = tiling;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  VIT_LAUNCH(h, VIT_PROF_OP, launch_linear_tc(p, h->dev_status, s));
+  VIT_LAUNCH(h, VIT_PROF_OP, launch_linear_tc(p, h->dev_status, s, &h->tmaps));
   return VIT_OK;
 }
 
@@ -691,7 +691,7 @@ int vit_op_attention(vit_handle* h, int dtype, int images, int T, int heads, int
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (dtype == VIT_BF16) {
     if (d % 16 || d > 128) return VIT_ERR_INVALID_ARG;
-    VIT_LAUNCH(h, VIT_PROF_ATTENTION, launch_attention_bf16((const bf16*)qkv, (bf16*)out, images, T, heads, d, h->dev_status, s));
+    VIT_LAUNCH(h, VIT_PROF_ATTENTION, launch_attention_bf16((const bf16*)qkv, (bf16*)out, images, T, heads, d, h->dev_status, s, &h->tmaps));
   } else if (dtype == VIT_FP32) {
     VIT_LAUNCH(h, VIT_PROF_ATTENTION, launch_attention_f32((const float*)qkv, (float*)out, images, T, heads, d, s));
   } else {

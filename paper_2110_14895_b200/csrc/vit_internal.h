@@ -1,11 +1,13 @@
 // Internal declarations shared by the library's translation units (not part of the C boundary).
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
 #include <stddef.h>
 #include <atomic>
 #include <mutex>
+#include <unordered_map>
 #include <vector>
 
 #include "../../include/vit.h"
@@ -57,6 +59,43 @@ struct LayerWeights {
   const float *qkv_c1, *qkv_c0, *fc1_c1, *fc1_c0;   // bf16 mode: the folded LayerNorm's column vectors (see EPI_LN_BIAS)
 };
 
+// Tensor maps are pure functions of (base address, extents, row pitch, box, swizzle).  The same
+// few maps recur on every call (weights always; activations as long as the caller reuses its
+// buffers), so a handle remembers them instead of asking the driver four to ten times per launch.
+struct TensorMapKey {
+  const void* base;
+  uint64_t rows, cols, ld;
+  uint32_t box_rows, box_cols, swizzle;
+  bool operator==(const TensorMapKey& o) const {
+    return base == o.base && rows == o.rows && cols == o.cols && ld == o.ld && box_rows == o.box_rows &&
+           box_cols == o.box_cols && swizzle == o.swizzle;
+  }
+};
+struct TensorMapKeyHash {
+  size_t operator()(const TensorMapKey& k) const {
+    uint64_t h = reinterpret_cast<uintptr_t>(k.base) * 0x9E3779B97F4A7C15ull;
+    for (uint64_t v : {k.rows, k.cols, k.ld, (uint64_t)k.box_rows, (uint64_t)k.box_cols, (uint64_t)k.swizzle})
+      h = (h ^ v) * 0x9E3779B97F4A7C15ull + (h >> 29);
+    return (size_t)h;
+  }
+};
+struct TensorMapCache {
+  std::mutex mu;
+  std::unordered_map<TensorMapKey, CUtensorMap, TensorMapKeyHash> maps;
+  // Returns the cached map or encodes it with `encode(CUtensorMap*) -> bool`.  cache == nullptr: always encode.
+  template <typename Encode>
+  static bool get(TensorMapCache* cache, const TensorMapKey& key, CUtensorMap* out, Encode encode) {
+    if (!cache) return encode(out);
+    std::lock_guard<std::mutex> lock(cache->mu);
+    auto it = cache->maps.find(key);
+    if (it != cache->maps.end()) { *out = it->second; return true; }
+    if (!encode(out)) return false;
+    if (cache->maps.size() >= 4096) cache->maps.clear();     // callers that never reuse buffers
+    cache->maps.emplace(key, *out);
+    return true;
+  }
+};
+
 struct ProfRecord { cudaEvent_t begin, end; int cls; };
 
 struct Handle {
@@ -76,21 +115,22 @@ struct Handle {
   std::atomic<uint64_t> launches;
   bool profiling;                    // event pair around every launch (single-threaded use)
   std::vector<ProfRecord> prof;
+  TensorMapCache tmaps;
 };
 
 // ---- kernel launchers (each returns a cudaError_t from the launch) ------------------------
 // bf16 family
 cudaError_t launch_layernorm_bf16(const bf16* x, const float* g, const float* b, float eps,
                                   bf16* y, int rows, int cols, cudaStream_t s);
-cudaError_t launch_linear_tc(const LinearArgs& a, int* dev_status, cudaStream_t s);   // tcgen05 GEMM
+cudaError_t launch_linear_tc(const LinearArgs& a, int* dev_status, cudaStream_t s, TensorMapCache* cache = nullptr);   // tcgen05 GEMM
 // per-row LayerNorm statistics: stats[r] = (mean, 1 / sqrt(biased variance + eps)) of x[r, :]
 cudaError_t launch_rowstats_bf16(const bf16* x, float eps, float2* stats, int rows, int cols, cudaStream_t s);
 // attention: the tcgen05 kernel where it supports the shape, else the warp-level mma kernel
 cudaError_t launch_attention_bf16(const bf16* qkv, bf16* out, int images, int T, int heads, int d,
-                                  int* dev_status, cudaStream_t s);
+                                  int* dev_status, cudaStream_t s, TensorMapCache* cache = nullptr);
 bool attention_tc_supported(int T, int d);
 cudaError_t launch_attention_tc(const bf16* qkv, bf16* out, int images, int T, int heads, int d,
-                                int* dev_status, cudaStream_t s);
+                                int* dev_status, cudaStream_t s, TensorMapCache* cache = nullptr);
 // fp32 family (SIMT)
 cudaError_t launch_layernorm_f32(const float* x, const float* g, const float* b, float eps,
                                  float* y, int rows, int cols, cudaStream_t s);

@@ -38,7 +38,7 @@ WORKLOADS = {
 }
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fc1 GEMM, from the ncu capture
 # whose summary is kept under profiles/ (same kernel build); None = not captured
-NCU_TRAFFIC = {"huge14": None}   # the fc1 epilogue changed since the last capture
+NCU_TRAFFIC = {"huge14": 384.4e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 NOMINAL_BF16_TFLOPS = 2250.0   # datasheet dense bf16 figure of the B200 (context; the measured peaks are the denominators)
 
@@ -350,6 +350,8 @@ def main():
     ap.add_argument("--mode", default="replicas", choices=["replicas", "pipeline"],
                     help="N > 1 only: independent replicas (default), or one pipeline stage per GPU with "
                          "point-to-point hand-off of the activations (the paper's runtime)")
+    ap.add_argument("--e2e-microbatch", type=int, default=64,
+                    help="microbatch of the host-buffer (end to end) leg: copies of one microbatch overlap the compute of others")
     ap.add_argument("--sweep", action="store_true",
                     help="also run the microbatch sweep (sizes 1..256, 4 stages, streams) and add it as 'sweep'")
     args = ap.parse_args()
@@ -435,7 +437,7 @@ def main():
     vit.vit_profile_enable(model.h, False)
 
     # end to end: host pixels in, host logits out, through the host-buffer entry point
-    e2e_mb = min(mb, 32)
+    e2e_mb = min(mb, args.e2e_microbatch)
     e2e_streams_n = min(4, max(1, batch // e2e_mb))
     e_wss, e_streams, e_wsb = model.make_pipeline_buffers(e2e_mb, e2e_streams_n)
     logits_host = torch.empty((batch, shape.num_classes), dtype=torch.float32).pin_memory()

@@ -1,5 +1,7 @@
 """End-to-end parity of the CUDA path with the CPU oracle on the same seeded inputs, and the
 stage-composition invariant on the GPU.  Everything goes through the C boundary."""
+import os
+
 import numpy as np
 import pytest
 
@@ -354,4 +356,32 @@ def test_pipeline_ragged_last_microbatch_and_argument_errors():
         m.run_pipeline([4], 2, dp, logits, wss, streams, 1024)     # workspace too small
     assert e.value.status == vit.VIT_ERR_WORKSPACE
     assert m.launches == before
+    m.close()
+
+
+def test_stage_pipeline_executor_on_the_gpu_single_rank():
+    """The stage-per-device runner with the CUDA executor on one rank (first and last stage at
+    once, so nothing is sent): embeds, runs the stage and classifies microbatch by microbatch, with
+    a ragged last microbatch, and gives the bits of a direct forward call."""
+    import torch.distributed as dist
+    from paper_2110_14895_b200 import pipeline as PL
+    shape = vitgen.preset("tiny16").with_(layers=3)
+    vit, m, params = _model(shape, _vit().VIT_BF16, 2)
+    port = 29000 + (os.getpid() % 500)
+    dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1)
+    try:
+        pipe = PL.StagePipeline(PL.VitStageExecutor(m, 0, shape.layers, True, True), dist, max_microbatch=2)
+        pix = torch.from_numpy(vitgen.make_pixels(shape, 5, seed=4)).cuda()
+        logits = torch.full((5, shape.num_classes), float("nan"), dtype=torch.float32, device="cuda")
+        for _ in range(2):                                   # two steps: the roll call advances
+            pipe.run(5, 2, pixels=pix, logits=logits)
+        torch.cuda.synchronize()
+        m.check()
+        assert [e for e in pipe.log if e[0] == "stage"][:3] == [("stage", 0), ("stage", 1), ("stage", 2)]
+        want = torch.cat([m.forward(pix[i:i + 2]) for i in (0, 2, 4)])
+        assert torch.equal(logits, want)
+        ok, msg = logits_within_tolerance(logits.cpu().numpy(), O.forward(params, shape, pix.cpu().numpy()), 2e-2, 0.9995)
+        assert ok, msg
+    finally:
+        dist.destroy_process_group()
     m.close()

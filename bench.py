@@ -529,7 +529,7 @@ def main():
         if sweep is not None:
             line["sweep"] = sweep
         if not args.no_cpu_baseline and world == 1:
-            n_img = 2 if preset == "huge14" else 4
+            n_img = 6 if preset == "huge14" else 16      # about 10-15 s of host work
             ips, cores, dt = oracle_images_per_s(shape, n_img)
             line["cpu_baseline"] = {"value": ips, "unit": "images/s", "cores": cores, "kind": "oracle",
                                     "sample": f"{n_img} images of the same workload, numpy fp64, {dt:.1f} s"}

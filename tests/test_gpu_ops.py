@@ -261,6 +261,44 @@ def test_attention_fp32(ctx, images, T, heads, d):
     assert np.abs(out.cpu().numpy() - want).max() <= 2e-5
 
 
+# ------------------------------------------------------------------------------- degenerate and extreme sizes
+def test_empty_inputs_launch_nothing_and_succeed(ctx):
+    """Zero rows / zero images are valid calls that do nothing (a ragged split can leave them)."""
+    vit, m = ctx
+    x = torch.zeros(64, 64, dtype=torch.bfloat16, device="cuda")
+    f = torch.zeros(64, dtype=torch.float32, device="cuda")
+    before = m.launches
+    vit.vit_op_linear(m.h, vit.VIT_BF16, 0, 64, 64, x.data_ptr(), x.data_ptr(), f.data_ptr(), 0, 0, x.data_ptr())
+    vit.vit_op_layernorm(m.h, vit.VIT_BF16, 0, 64, x.data_ptr(), f.data_ptr(), f.data_ptr(), 1e-6, x.data_ptr())
+    vit.vit_op_rowstats(m.h, 0, 64, x.data_ptr(), 1e-6, f.data_ptr())
+    vit.vit_op_attention(m.h, vit.VIT_BF16, 0, 197, 1, 64, x.data_ptr(), x.data_ptr())
+    m.check()
+    assert (x == 0).all() and (f == 0).all()
+    assert m.launches - before <= 4          # counted as calls; no kernel had anything to do
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 8, 8), (3, 16, 24), (130, 8, 4096)])
+def test_linear_bf16_smallest_and_longest_shapes(ctx, M, N, K):
+    _linear_case(ctx, M, N, K, 0, 0)
+    _linear_case(ctx, M, N, K, 2, 0)
+
+
+def test_attention_bf16_longest_sequence(ctx):
+    """T = 512 is the longest sequence a configuration may have (warp-level kernel)."""
+    vit, m = ctx
+    rng = np.random.default_rng(512)
+    T, heads, d = 512, 2, 64
+    H = heads * d
+    qkv, qr = _bf16(rng.normal(size=(T, 3 * H)))
+    out = torch.full((T, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+    vit.vit_op_attention(m.h, vit.VIT_BF16, 1, T, heads, d, qkv.data_ptr(), out.data_ptr())
+    m.check()
+    want = _oracle_attention(qr, 1, T, heads)
+    got = out.float().cpu().numpy()
+    assert np.isfinite(got).all()
+    assert np.abs(got - want).max() <= 2 * BF16_EPS * np.abs(want).max() + 5e-4 * np.abs(qr[:, 2 * H:]).max()
+
+
 # ------------------------------------------------------------------------------- argument checks
 def test_op_argument_errors(ctx):
     vit, m = ctx

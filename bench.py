@@ -353,7 +353,8 @@ def main():
     ap.add_argument("--e2e-microbatch", type=int, default=64,
                     help="microbatch of the host-buffer (end to end) leg: copies of one microbatch overlap the compute of others")
     ap.add_argument("--sweep", action="store_true",
-                    help="also run the microbatch sweep (sizes 1..256, 4 stages, streams) and add it as 'sweep'")
+                    help="run the microbatch sweep (sizes 1..256, 4 stages, streams; key 'sweep') also for workloads other than the default")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the microbatch sweep of the default run")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "b200" else args.warmup
 
@@ -382,8 +383,7 @@ def main():
     shape = vitgen.preset(preset)
     counts = stage_counts(shape, n_stages)
     _, blob = vitgen.make_params(shape, seed=0)
-    model = vit.VitModel(shape, blob, vit.VIT_BF16, max(mb, 256) if args.sweep else mb, device=dev)
-    del blob
+    model = vit.VitModel(shape, blob, vit.VIT_BF16, mb, device=dev)
     pix_host = torch.from_numpy(vitgen.make_pixels(shape, batch, seed=rank_pixel_seed(rank))).pin_memory()
     pix = pix_host.to(dev)
     logits = torch.empty((batch, shape.num_classes), dtype=torch.float32, device=dev)
@@ -453,9 +453,14 @@ def main():
         model.check(s)
     e2e_value = aggregate_images_per_s(world, batch, ms_e2e)
 
+    # microbatch sweep (ViT-H/14 by default): a handle of its own with room for microbatches of 256,
+    # after the headline measurements so that they are not affected
     sweep = None
-    if args.sweep:
-        sweep = microbatch_sweep(vit, model, shape, dev, torch)
+    if world == 1 and not args.no_sweep and (args.sweep or args.workload == "huge14"):
+        sweep_model = vit.VitModel(shape, blob, vit.VIT_BF16, 256, device=dev)
+        sweep = microbatch_sweep(vit, sweep_model, shape, dev, torch)
+        sweep_model.close()
+    del blob
 
     # the other single-GPU configurations of the metric, briefly (rank 0 of a single-GPU run only)
     extra = {}

@@ -383,8 +383,16 @@ __global__ void im2col_kernel(const float* __restrict__ px, TOut* __restrict__ c
       }
     }
     TOut* o = cols + row * k_pad + q * 8;
+    if (sizeof(TOut) == 2) {                      // bf16: the eight columns as one 16-byte store
+      uint4 w;
+      __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&w);
 #pragma unroll
-    for (int e = 0; e < 8; ++e) o[e] = (TOut)v[e];
+      for (int e = 0; e < 4; ++e) h2[e] = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
+      *reinterpret_cast<uint4*>(o) = w;
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) o[e] = (TOut)v[e];
+    }
   }
 }
 

@@ -385,3 +385,37 @@ def test_stage_pipeline_executor_on_the_gpu_single_rank():
     finally:
         dist.destroy_process_group()
     m.close()
+
+
+@pytest.mark.parametrize("name,mb", [("tiny16", 3), ("deit_tiny16", 2), ("huge14", 2)])
+def test_kernels_stay_inside_their_buffers(name, mb):
+    """Workspace, activations and logits are carved out of one allocation with guard bands of a
+    known pattern on both sides of each; after patch embed, two stages and the head every guard
+    byte is still in place (with exactly the workspace size the library asks for)."""
+    shape = vitgen.preset(name).with_(layers=2)
+    vit, m, _ = _model(shape, _vit().VIT_BF16, mb)
+    G = 4096                                                     # guard bytes, keeps 256-byte alignment
+    sizes = {"ws": vit.vit_workspace_bytes(m.cfg, mb), "tok": mb * m.T * shape.hidden * 2,
+             "out": mb * m.T * shape.hidden * 2, "logits": mb * shape.num_classes * 4}
+    off, total = {}, G
+    for k, n in sizes.items():
+        off[k] = total
+        total += (n + 255) // 256 * 256 + G
+    buf = torch.full((total,), 0xA5, dtype=torch.uint8, device="cuda")
+    base = buf.data_ptr()
+    assert base % 256 == 0
+    pix = torch.from_numpy(vitgen.make_pixels(shape, mb, seed=1)).cuda()
+    ptr = {k: base + o for k, o in off.items()}
+    vit.vit_patch_embed(m.h, mb, pix.data_ptr(), ptr["tok"], ptr["ws"], sizes["ws"])
+    vit.vit_run_stage(m.h, 0, 1, mb, ptr["tok"], ptr["out"], ptr["ws"], sizes["ws"])
+    vit.vit_run_stage(m.h, 1, 2, mb, ptr["out"], ptr["out"], ptr["ws"], sizes["ws"])
+    vit.vit_head(m.h, mb, ptr["out"], ptr["logits"], ptr["ws"], sizes["ws"])
+    m.check()
+    host = buf.cpu().numpy()
+    guards = np.ones(total, dtype=bool)
+    for k, n in sizes.items():
+        guards[off[k]:off[k] + n] = False
+    assert (host[guards] == 0xA5).all(), {k: int((host[off[k] + sizes[k]:off[k] + sizes[k] + G] != 0xA5).sum()) for k in sizes}
+    logits = host[off["logits"]:off["logits"] + sizes["logits"]].copy().view(np.float32)
+    assert np.isfinite(logits).all()
+    m.close()
